@@ -1,0 +1,300 @@
+// Gradients of O = softmax(scale Q K^g^T) V^g + LCE(V) for a fixed routing
+// index (Eq. 7 with Eq. 1; the index of Eq. 5 is a constant), fp32 arithmetic
+// on CUDA cores.  Every sum has a fixed order: no atomics on the data path.
+//
+//   1. inverse index: for each key region, the list (in (query region, slot)
+//      order) of query regions that routed to it, as CSR.
+//   2. dQ kernel, one thread per (query, head): delta = rowsum(P o dP), then
+//      dQ = scale * sum_j P_j (dP_j - delta) K_j; delta is kept for step 3.
+//   3. dK/dV kernel, one thread per (key token, head): walks the inverse index,
+//      recomputes P from the saved log-sum-exp, accumulates dK, dV, then adds
+//      the LCE adjoint dV += sum_ij w[c,i,j] dO[y-i+2, x-j+2, c].
+//   4. d_lce_w / d_lce_b: per-CTA partial sums, then a fixed-order final sum.
+#include "bra_internal.h"
+
+namespace bra {
+
+// ------------------------------------------------------------ inverse index
+// grid: B * heads_i CTAs; block: R threads rounded up to a warp.
+__global__ void inverse_index_kernel(const int32_t* __restrict__ index, int32_t* __restrict__ inv_off,
+                                     int32_t* __restrict__ inv_list, Dims dm) {
+    extern __shared__ int32_t sm[];   // counts[R + 1]
+    const int bh = blockIdx.x;
+    const int32_t* idx = index + (size_t)bh * dm.R * dm.topk;
+    const int entries = dm.R * dm.topk;
+    const int j = threadIdx.x;
+    int count = 0;
+    if (j < dm.R)
+        for (int e = 0; e < entries; ++e) count += (idx[e] == j);
+    if (j < dm.R) sm[j] = count;
+    __syncthreads();
+    if (j == 0) {
+        int run = 0;
+        for (int r = 0; r < dm.R; ++r) { const int c = sm[r]; sm[r] = run; run += c; }
+        sm[dm.R] = run;
+    }
+    __syncthreads();
+    int32_t* off = inv_off + (size_t)bh * (dm.R + 1);
+    if (j <= dm.R) off[j] = sm[j];
+    if (j < dm.R) {
+        int32_t* out = inv_list + (size_t)bh * entries + sm[j];
+        for (int e = 0; e < entries; ++e)
+            if (idx[e] == j) *out++ = e / dm.topk;      // the query region of entry e
+    }
+}
+
+// ------------------------------------------------------------ dQ and delta
+template <typename T, int D>
+__global__ void __launch_bounds__(128)
+bwd_dq_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __restrict__ V,
+              const int32_t* __restrict__ index, const float* __restrict__ lse,
+              const T* __restrict__ dO, T* __restrict__ dQ, float* __restrict__ delta,
+              int32_t* __restrict__ status, Dims dm) {
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long total = (long long)dm.B * dm.heads * dm.R * dm.n_r;
+    if (gid >= total) return;
+    const int t = (int)(gid % dm.n_r);
+    const int i = (int)((gid / dm.n_r) % dm.R);
+    const int h = (int)((gid / ((long long)dm.n_r * dm.R)) % dm.heads);
+    const int b = (int)(gid / ((long long)dm.n_r * dm.R * dm.heads));
+    const int y = (i / dm.S) * dm.hs + t / dm.ws;
+    const int x = (i % dm.S) * dm.ws + t % dm.ws;
+    const size_t img = (size_t)b * dm.N * dm.C;
+    const size_t tok = img + ((size_t)y * dm.W + x) * dm.C + (size_t)h * D;
+    const size_t stat = ((size_t)b * dm.heads + h) * dm.N + (size_t)y * dm.W + x;
+
+    float q[D], go[D], acc[D];
+    load_row<D>(Q + tok, q);
+    load_row<D>(dO + tok, go);
+#pragma unroll
+    for (int c = 0; c < D; ++c) { q[c] *= dm.scale; acc[c] = 0.f; }
+    const float l = lse[stat];
+    const int hi = dm.heads_i == 1 ? 0 : h;
+    const int32_t* row = index + (((size_t)b * dm.heads_i + hi) * dm.R + i) * dm.topk;
+
+    float dsum = 0.f;
+    for (int pass = 0; pass < 2; ++pass) {
+        for (int m = 0; m < dm.topk; ++m) {
+            const int r = row[m];
+            if (r < 0 || r >= dm.R) { record_error(status, BRA_ERR_INDEX, r); continue; }
+            const int y0 = (r / dm.S) * dm.hs, x0 = (r % dm.S) * dm.ws;
+            for (int j = 0; j < dm.n_r; ++j) {
+                const size_t kt = img + ((size_t)(y0 + j / dm.ws) * dm.W + x0 + j % dm.ws) * dm.C + (size_t)h * D;
+                float kr[D], vr[D];
+                load_row<D>(K + kt, kr);
+                load_row<D>(V + kt, vr);
+                float s = 0.f, dp = 0.f;
+#pragma unroll
+                for (int c = 0; c < D; ++c) { s = fmaf(q[c], kr[c], s); dp = fmaf(go[c], vr[c], dp); }
+                const float p = expf(s - l);
+                if (pass == 0) {
+                    dsum = fmaf(p, dp, dsum);
+                } else {
+                    const float ds = p * (dp - dsum);
+#pragma unroll
+                    for (int c = 0; c < D; ++c) acc[c] = fmaf(ds, kr[c], acc[c]);
+                }
+            }
+        }
+    }
+    delta[stat] = dsum;
+#pragma unroll
+    for (int c = 0; c < D; ++c) acc[c] *= dm.scale;
+    store_row<D>(dQ + tok, acc);
+}
+
+// ------------------------------------------------------------ dK, dV
+template <typename T, int D>
+__global__ void __launch_bounds__(128)
+bwd_dkv_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __restrict__ V,
+               const int32_t* __restrict__ inv_off, const int32_t* __restrict__ inv_list,
+               const float* __restrict__ lse, const float* __restrict__ delta,
+               const T* __restrict__ dO, const float* __restrict__ lce_w,
+               T* __restrict__ dK, T* __restrict__ dV, Dims dm) {
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long total = (long long)dm.B * dm.heads * dm.R * dm.n_r;
+    if (gid >= total) return;
+    const int t = (int)(gid % dm.n_r);
+    const int jr = (int)((gid / dm.n_r) % dm.R);          // key region
+    const int h = (int)((gid / ((long long)dm.n_r * dm.R)) % dm.heads);
+    const int b = (int)(gid / ((long long)dm.n_r * dm.R * dm.heads));
+    const int y = (jr / dm.S) * dm.hs + t / dm.ws;
+    const int x = (jr % dm.S) * dm.ws + t % dm.ws;
+    const size_t img = (size_t)b * dm.N * dm.C;
+    const size_t tok = img + ((size_t)y * dm.W + x) * dm.C + (size_t)h * D;
+
+    float kr[D], vr[D], gk[D], gv[D];
+    load_row<D>(K + tok, kr);
+    load_row<D>(V + tok, vr);
+#pragma unroll
+    for (int c = 0; c < D; ++c) { kr[c] *= dm.scale; gk[c] = 0.f; gv[c] = 0.f; }
+
+    const int hi = dm.heads_i == 1 ? 0 : h;
+    const size_t bh = (size_t)b * dm.heads_i + hi;
+    const int32_t* off = inv_off + bh * (dm.R + 1);
+    const int32_t* list = inv_list + bh * dm.R * dm.topk;
+    const size_t stat0 = ((size_t)b * dm.heads + h) * dm.N;
+    for (int e = off[jr]; e < off[jr + 1]; ++e) {
+        const int i = list[e];                            // a query region that lists jr
+        const int y0 = (i / dm.S) * dm.hs, x0 = (i % dm.S) * dm.ws;
+        for (int tq = 0; tq < dm.n_r; ++tq) {
+            const int yq = y0 + tq / dm.ws, xq = x0 + tq % dm.ws;
+            const size_t qt = img + ((size_t)yq * dm.W + xq) * dm.C + (size_t)h * D;
+            float qr[D], go[D];
+            load_row<D>(Q + qt, qr);
+            load_row<D>(dO + qt, go);
+            float s = 0.f, dp = 0.f;
+#pragma unroll
+            for (int c = 0; c < D; ++c) { s = fmaf(qr[c], kr[c], s); dp = fmaf(go[c], vr[c], dp); }
+            const size_t st = stat0 + (size_t)yq * dm.W + xq;
+            const float p = expf(s - lse[st]);
+            const float ds = p * (dp - delta[st]);
+#pragma unroll
+            for (int c = 0; c < D; ++c) { gk[c] = fmaf(ds, qr[c], gk[c]); gv[c] = fmaf(p, go[c], gv[c]); }
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < D; ++c) gk[c] *= dm.scale;
+    if (dm.lce) {
+        const float* wh = lce_w + (size_t)h * D * 25;
+        for (int ti = 0; ti < 5; ++ti) {
+            const int yy = y - ti + 2;
+            if (yy < 0 || yy >= dm.H) continue;
+            for (int tj = 0; tj < 5; ++tj) {
+                const int xx = x - tj + 2;
+                if (xx < 0 || xx >= dm.W) continue;
+                float go[D];
+                load_row<D>(dO + img + ((size_t)yy * dm.W + xx) * dm.C + (size_t)h * D, go);
+#pragma unroll
+                for (int c = 0; c < D; ++c) gv[c] = fmaf(__ldg(wh + c * 25 + ti * 5 + tj), go[c], gv[c]);
+            }
+        }
+    }
+    store_row<D>(dK + tok, gk);
+    store_row<D>(dV + tok, gv);
+}
+
+// ------------------------------------------------------------ d_lce_w, d_lce_b
+// Partial sums: CTA p covers a contiguous range of (image, row) pairs; thread c
+// (one per channel, looped) keeps the 25 tap sums and the bias sum of its channel.
+template <typename T>
+__global__ void __launch_bounds__(256)
+bwd_dw_partial_kernel(const T* __restrict__ V, const T* __restrict__ dO, float* __restrict__ part,
+                      int rows_per_block, Dims dm) {
+    const long long rows = (long long)dm.B * dm.H;
+    const long long r0 = (long long)blockIdx.x * rows_per_block;
+    const long long r1 = r0 + rows_per_block < rows ? r0 + rows_per_block : rows;
+    for (int c = threadIdx.x; c < dm.C; c += blockDim.x) {
+        float acc[26];
+#pragma unroll
+        for (int k = 0; k < 26; ++k) acc[k] = 0.f;
+        for (long long r = r0; r < r1; ++r) {
+            const int b = (int)(r / dm.H), y = (int)(r % dm.H);
+            const size_t img = (size_t)b * dm.N * dm.C;
+            for (int x = 0; x < dm.W; ++x) {
+                const float g = (float)dO[img + ((size_t)y * dm.W + x) * dm.C + c];
+                acc[25] += g;
+#pragma unroll
+                for (int ti = 0; ti < 5; ++ti) {
+                    const int yy = y + ti - 2;
+                    if (yy < 0 || yy >= dm.H) continue;
+#pragma unroll
+                    for (int tj = 0; tj < 5; ++tj) {
+                        const int xx = x + tj - 2;
+                        if (xx < 0 || xx >= dm.W) continue;
+                        acc[ti * 5 + tj] = fmaf(g, (float)V[img + ((size_t)yy * dm.W + xx) * dm.C + c], acc[ti * 5 + tj]);
+                    }
+                }
+            }
+        }
+        float* out = part + ((size_t)blockIdx.x * dm.C + c) * 26;
+#pragma unroll
+        for (int k = 0; k < 26; ++k) out[k] = acc[k];
+    }
+}
+
+__global__ void bwd_dw_final_kernel(const float* __restrict__ part, int blocks,
+                                    float* __restrict__ d_lce_w, float* __restrict__ d_lce_b, Dims dm) {
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;   // (channel, slot)
+    if (o >= dm.C * 26) return;
+    float s = 0.f;
+    for (int p = 0; p < blocks; ++p) s += part[(size_t)p * dm.C * 26 + o];
+    const int c = o / 26, k = o % 26;
+    if (k < 25) { if (d_lce_w) d_lce_w[c * 25 + k] = s; }
+    else if (d_lce_b) d_lce_b[c] = s;
+}
+
+bool backward_supported(const Dims& d) {
+    return (d.d == 16 || d.d == 32 || d.d == 64) && d.R <= 1000;
+}
+
+template <typename T, int D>
+static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, const void* V,
+                                const int32_t* index, const float* lce_w, const float* lse,
+                                const void* dO, void* dQ, void* dK, void* dV,
+                                float* d_lce_w, float* d_lce_b, char* ws, const WsLayout& L,
+                                cudaStream_t st) {
+    int32_t* status = reinterpret_cast<int32_t*>(ws + L.status);
+    float* delta = reinterpret_cast<float*>(ws + L.delta);
+    int32_t* inv_off = reinterpret_cast<int32_t*>(ws + L.inv_off);
+    int32_t* inv_list = reinterpret_cast<int32_t*>(ws + L.inv_list);
+    float* part = reinterpret_cast<float*>(ws + L.dw_part);
+    const T* q = static_cast<const T*>(Q); const T* k = static_cast<const T*>(K);
+    const T* v = static_cast<const T*>(V); const T* go = static_cast<const T*>(dO);
+    cudaError_t e;
+
+    const int thr = (d.R + 1 + 31) / 32 * 32;
+    inverse_index_kernel<<<d.B * d.heads_i, thr, sizeof(int32_t) * (d.R + 1), st>>>(index, inv_off, inv_list, d);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+
+    const long long total = (long long)d.B * d.heads * d.R * d.n_r;
+    const unsigned blocks = (unsigned)((total + 127) / 128);
+    bwd_dq_kernel<T, D><<<blocks, 128, 0, st>>>(q, k, v, index, lse, go, static_cast<T*>(dQ), delta, status, d);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+
+    bwd_dkv_kernel<T, D><<<blocks, 128, 0, st>>>(q, k, v, inv_off, inv_list, lse, delta, go, lce_w,
+                                                 static_cast<T*>(dK), static_cast<T*>(dV), d);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+
+    if (d.lce || d_lce_b) {
+        const long long rows = (long long)d.B * d.H;
+        const int rpb = (int)((rows + L.dw_blocks - 1) / L.dw_blocks);
+        const int nblk = (int)((rows + rpb - 1) / rpb);
+        bwd_dw_partial_kernel<T><<<nblk, d.C < 256 ? (d.C + 31) / 32 * 32 : 256, 0, st>>>(v, go, part, rpb, d);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        bwd_dw_final_kernel<<<(d.C * 26 + 127) / 128, 128, 0, st>>>(part, nblk, d.lce ? d_lce_w : nullptr, d_lce_b, d);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+template <typename T>
+static cudaError_t launch_bwd_d(const Dims& d, const void* Q, const void* K, const void* V,
+                                const int32_t* index, const float* lce_w, const float* lse,
+                                const void* dO, void* dQ, void* dK, void* dV,
+                                float* d_lce_w, float* d_lce_b, char* ws, const WsLayout& L,
+                                cudaStream_t st) {
+    switch (d.d) {
+        case 16: return launch_bwd_t<T, 16>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+        case 32: return launch_bwd_t<T, 32>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+        case 64: return launch_bwd_t<T, 64>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_backward(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
+                            const int32_t* index, const float* lce_w, const float* lse,
+                            const void* dO, void* dQ, void* dK, void* dV,
+                            float* d_lce_w, float* d_lce_b,
+                            char* ws, const WsLayout& L, cudaStream_t st) {
+    if (dtype == BRA_BF16)
+        return launch_bwd_d<__nv_bfloat16>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+    return launch_bwd_d<float>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+}
+
+}  // namespace bra

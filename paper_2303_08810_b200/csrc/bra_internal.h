@@ -1,0 +1,125 @@
+// Internal declarations shared by the translation units of the BRA library.
+// Nothing here is part of the C boundary (include/bra.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/bra.h"
+
+namespace bra {
+
+// Problem with every derived quantity the kernels need, passed by value.
+struct Dims {
+    int B, H, W, C, heads, S, topk;
+    int d;        // C / heads
+    int R;        // S * S regions
+    int hs, ws;   // region height / width in tokens
+    int n_r;      // hs * ws tokens per region
+    int N;        // H * W tokens per image
+    int heads_i;  // heads of the routing index: heads, or 1 with shared routing
+    int lce;      // 1: add LCE
+    float scale;  // softmax scale (Eq. 1)
+};
+
+// Scratch layout (byte offsets from ws, all multiples of 256).
+struct WsLayout {
+    size_t status;      // int32[64]: [0] first device error, [1] detail
+    size_t q_mean;      // fp32 [B,R,C]
+    size_t k_mean;      // fp32 [B,R,C]
+    size_t index;       // int32 [B,heads_i,R,topk] (bra_forward with index == NULL)
+    size_t delta;       // fp32 [B,heads,N]  rowsum(P o dP) of the backward pass
+    size_t inv_off;     // int32 [B,heads_i,R+1] CSR offsets of the inverse routing index
+    size_t inv_list;    // int32 [B,heads_i,R*topk] query regions routed to each key region
+    size_t dw_part;     // fp32 [dw_blocks, C*26] partial LCE weight / bias gradients
+    size_t total;
+    int dw_blocks;
+};
+
+WsLayout ws_layout(const Dims& d);
+
+// Host-side bookkeeping of kernel launches for bra_last_launch_count().
+void count_launch(int n = 1);
+
+// ---- kernel launchers (each returns the cudaError of its launches) ----------
+cudaError_t launch_pool(const Dims& d, int dtype, const void* Q, const void* K,
+                        float* q_mean, float* k_mean, cudaStream_t st);
+cudaError_t launch_route(const Dims& d, const float* q_mean, const float* k_mean,
+                         int32_t* index, cudaStream_t st);
+// true if this build has a routing kernel for the problem
+bool route_supported(const Dims& d);
+
+bool attend_simt_supported(const Dims& d);
+cudaError_t launch_attend_simt(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
+                               const int32_t* index, const float* lce_w, const float* lce_b,
+                               void* O, float* lse, int32_t* status, cudaStream_t st);
+
+bool attend_mma_supported(const Dims& d, int dtype);
+cudaError_t launch_attend_mma(const Dims& d, const void* Q, const void* K, const void* V,
+                              const int32_t* index, const float* lce_w, const float* lce_b,
+                              void* O, float* lse, int32_t* status, cudaStream_t st);
+
+bool attend_tc_supported(const Dims& d, int dtype);
+cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const void* V,
+                             const int32_t* index, const float* lce_w, const float* lce_b,
+                             void* O, float* lse, int32_t* status, cudaStream_t st);
+
+bool backward_supported(const Dims& d);
+cudaError_t launch_backward(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
+                            const int32_t* index, const float* lce_w, const float* lse,
+                            const void* dO, void* dQ, void* dK, void* dV,
+                            float* d_lce_w, float* d_lce_b,
+                            char* ws, const WsLayout& L, cudaStream_t st);
+
+// ---- device helpers -----------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ void record_error(int32_t* status, int code, int detail) {
+    if (atomicCAS(status, 0, code) == 0) status[1] = detail;
+}
+
+// Load `n` consecutive elements (n multiple of 8 for bf16 / 4 for fp32, 16-byte aligned) as fp32.
+template <int n>
+__device__ __forceinline__ void load_row(const float* __restrict__ p, float* out) {
+#pragma unroll
+    for (int i = 0; i < n; i += 4) {
+        float4 v = __ldg(reinterpret_cast<const float4*>(p + i));
+        out[i] = v.x; out[i + 1] = v.y; out[i + 2] = v.z; out[i + 3] = v.w;
+    }
+}
+template <int n>
+__device__ __forceinline__ void load_row(const __nv_bfloat16* __restrict__ p, float* out) {
+#pragma unroll
+    for (int i = 0; i < n; i += 8) {
+        uint4 v = __ldg(reinterpret_cast<const uint4*>(p + i));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            out[i + 2 * j] = __uint_as_float(w[j] << 16);
+            out[i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+        }
+    }
+}
+template <int n>
+__device__ __forceinline__ void store_row(float* p, const float* v) {
+#pragma unroll
+    for (int i = 0; i < n; i += 4)
+        *reinterpret_cast<float4*>(p + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+}
+template <int n>
+__device__ __forceinline__ void store_row(__nv_bfloat16* p, const float* v) {
+#pragma unroll
+    for (int i = 0; i < n; i += 8) {
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(v[i + 2 * j], v[i + 2 * j + 1]);
+            w[j] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(p + i) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+#endif  // __CUDACC__
+
+}  // namespace bra

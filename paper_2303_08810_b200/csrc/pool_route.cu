@@ -1,0 +1,216 @@
+// Region-to-region routing (Section 3.2): per-region average of Q and K,
+// region affinity A^r = Q^r (K^r)^T (Eq. 4) and row-wise top-k index (Eq. 5).
+#include "bra_internal.h"
+
+namespace bra {
+
+// ------------------------------------------------------------------ pooling
+// One CTA reduces one row of regions of one image of one tensor: the hs x W x C
+// strip of tokens it covers is contiguous in memory.  Each thread owns
+// (column x, 16-byte channel vector) pairs, sums the hs rows in registers with
+// independent 16-byte loads, parks the partial sums in shared memory, and the
+// CTA then folds the ws columns of every region.
+template <typename T> struct Vec;
+template <> struct Vec<float> { static constexpr int n = 4; };
+template <> struct Vec<__nv_bfloat16> { static constexpr int n = 8; };
+
+template <typename T>
+__global__ void __launch_bounds__(1024)
+pool_kernel(const T* __restrict__ Q, const T* __restrict__ K,
+            float* __restrict__ q_mean, float* __restrict__ k_mean, Dims dm) {
+    constexpr int VEC = Vec<T>::n;
+    extern __shared__ float part[];   // [W][C]
+    const int ry = blockIdx.x, b = blockIdx.y;
+    const T* src = blockIdx.z == 0 ? Q : K;
+    float* dst = blockIdx.z == 0 ? q_mean : k_mean;
+    const int cvecs = dm.C / VEC;
+    const int items = dm.W * cvecs;
+    const size_t row_elems = (size_t)dm.W * dm.C;
+    const T* strip = src + ((size_t)b * dm.H + (size_t)ry * dm.hs) * row_elems;
+
+    for (int it = threadIdx.x; it < items; it += blockDim.x) {
+        float acc[VEC];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
+        const T* p = strip + (size_t)it * VEC;      // (x, cvec) in row 0 of the strip
+        int y = 0;
+        for (; y + 4 <= dm.hs; y += 4) {            // four loads in flight
+            float v[4][VEC];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) load_row<VEC>(p + (size_t)(y + u) * row_elems, v[u]);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) acc[i] += v[u][i];
+        }
+        for (; y < dm.hs; ++y) {
+            float v[VEC];
+            load_row<VEC>(p + (size_t)y * row_elems, v);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) acc[i] += v[i];
+        }
+#pragma unroll
+        for (int i = 0; i < VEC; i += 4)
+            *reinterpret_cast<float4*>(&part[it * VEC + i]) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+    }
+    __syncthreads();
+    const float inv = 1.0f / (float)dm.n_r;
+    for (int o = threadIdx.x; o < dm.S * dm.C; o += blockDim.x) {
+        const int rx = o / dm.C, c = o - rx * dm.C;
+        float s = 0.f;
+        for (int x = 0; x < dm.ws; ++x) s += part[(rx * dm.ws + x) * dm.C + c];
+        dst[((size_t)b * dm.R + ry * dm.S + rx) * dm.C + c] = s * inv;
+    }
+}
+
+cudaError_t launch_pool(const Dims& d, int dtype, const void* Q, const void* K,
+                        float* q_mean, float* k_mean, cudaStream_t st) {
+    const int vec = dtype == BRA_BF16 ? 8 : 4;
+    int items = d.W * (d.C / vec);
+    int threads = ((items < 1024 ? items : 1024) + 31) / 32 * 32;
+    size_t smem = sizeof(float) * (size_t)d.W * d.C;
+    dim3 grid(d.S, d.B, 2);
+    cudaError_t e;
+    if (dtype == BRA_BF16) {
+        if (smem > 48 * 1024 &&
+            (e = cudaFuncSetAttribute(pool_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
+            return e;
+        pool_kernel<__nv_bfloat16><<<grid, threads, smem, st>>>(
+            static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K), q_mean, k_mean, d);
+    } else {
+        if (smem > 48 * 1024 &&
+            (e = cudaFuncSetAttribute(pool_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
+            return e;
+        pool_kernel<float><<<grid, threads, smem, st>>>(
+            static_cast<const float*>(Q), static_cast<const float*>(K), q_mean, k_mean, d);
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ routing
+// One CTA per (image, routing head).  K^r of the head sits in shared memory
+// (row stride odd, so a warp reading one row per lane has no bank conflict).
+// One warp per affinity row: lane l holds the scores of regions l, l+32, ...;
+// the row is sorted by a warp-wide bitonic network on 64-bit keys
+//   (order-preserving bits of the fp32 score) << 32 | (0xffffffff - region)
+// descending, which yields score-descending, lower-region-first order.
+__device__ __forceinline__ uint32_t ordered_bits(float s) {
+    s += 0.0f;                                  // -0 -> +0: equal scores tie on the index
+    uint32_t u = __float_as_uint(s);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+template <int E>   // E score slots per lane: handles R <= 32 * E
+__global__ void __launch_bounds__(256)
+route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
+             int32_t* __restrict__ index, Dims dm) {
+    extern __shared__ float ks[];               // [R][dc + 1]
+    const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
+    const int dc = dm.heads_i == 1 ? dm.C : dm.d;   // channels the affinity sums over
+    const int c0 = dm.heads_i == 1 ? 0 : h * dm.d;
+    const int ld = dc + 1;
+    const float* kb = k_mean + (size_t)b * dm.R * dm.C + c0;
+    for (int i = threadIdx.x; i < dm.R * dc; i += blockDim.x) {
+        const int r = i / dc, c = i - r * dc;
+        ks[r * ld + c] = kb[(size_t)r * dm.C + c];
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int i = warp; i < dm.R; i += nwarps) {
+        const float* qrow = q_mean + ((size_t)b * dm.R + i) * dm.C + c0;
+        float acc[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] = 0.f;
+        for (int cb = 0; cb < dc; cb += 32) {
+            const float qv = (cb + lane < dc) ? qrow[cb + lane] : 0.f;
+            const int lim = dc - cb < 32 ? dc - cb : 32;
+            for (int c = 0; c < lim; ++c) {
+                const float qc = __shfl_sync(0xffffffffu, qv, c);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const int j = lane + 32 * e;
+                    if (j < dm.R) acc[e] = fmaf(qc, ks[j * ld + cb + c], acc[e]);
+                }
+            }
+        }
+        unsigned long long key[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int j = lane + 32 * e;
+            key[e] = j < dm.R ? ((unsigned long long)ordered_bits(acc[e]) << 32) | (0xffffffffu - (uint32_t)j)
+                              : 0ull;
+        }
+        // bitonic sort, descending, element id = slot * 32 + lane
+#pragma unroll
+        for (int k2 = 2; k2 <= 32 * E; k2 <<= 1) {
+#pragma unroll
+            for (int j = k2 >> 1; j > 0; j >>= 1) {
+                if (j >= 32) {
+                    const int js = j >> 5;
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        if ((e & js) == 0) {
+                            const int id = e * 32 + lane;
+                            const bool desc = (id & k2) == 0;
+                            unsigned long long a = key[e], c = key[e | js];
+                            const bool swap = desc ? (a < c) : (a > c);
+                            key[e] = swap ? c : a;
+                            key[e | js] = swap ? a : c;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        const int id = e * 32 + lane;
+                        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key[e], j);
+                        const bool lower = (id & j) == 0;
+                        const bool desc = (id & k2) == 0;
+                        const bool keep_max = lower == desc;
+                        const unsigned long long mx = key[e] > other ? key[e] : other;
+                        const unsigned long long mn = key[e] > other ? other : key[e];
+                        key[e] = keep_max ? mx : mn;
+                    }
+                }
+            }
+        }
+        int32_t* out = index + (((size_t)b * dm.heads_i + h) * dm.R + i) * dm.topk;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int rank = e * 32 + lane;
+            if (rank < dm.topk) out[rank] = (int32_t)(0xffffffffu - (uint32_t)(key[e] & 0xffffffffull));
+        }
+    }
+}
+
+static size_t route_smem(const Dims& d) {
+    const int dc = d.heads_i == 1 ? d.C : d.d;
+    return sizeof(float) * (size_t)d.R * (dc + 1);
+}
+
+bool route_supported(const Dims& d) {
+    return d.R <= 256 && route_smem(d) <= 200 * 1024 && sizeof(float) * (size_t)d.W * d.C <= 200 * 1024;
+}
+
+template <int E>
+static cudaError_t launch_route_e(const Dims& d, const float* q_mean, const float* k_mean,
+                                  int32_t* index, cudaStream_t st) {
+    const size_t smem = route_smem(d);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(route_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    route_kernel<E><<<d.B * d.heads_i, 256, smem, st>>>(q_mean, k_mean, index, d);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_route(const Dims& d, const float* q_mean, const float* k_mean,
+                         int32_t* index, cudaStream_t st) {
+    if (d.R <= 32) return launch_route_e<1>(d, q_mean, k_mean, index, st);
+    if (d.R <= 64) return launch_route_e<2>(d, q_mean, k_mean, index, st);
+    if (d.R <= 128) return launch_route_e<4>(d, q_mean, k_mean, index, st);
+    return launch_route_e<8>(d, q_mean, k_mean, index, st);
+}
+
+}  // namespace bra

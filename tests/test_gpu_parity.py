@@ -1,0 +1,298 @@
+"""GPU parity: the CUDA path, through the C boundary, against the fp64 CPU oracle
+on the same seeded inputs.
+
+Tolerances (stated by the benchmark definition):
+  * routing index: bit-exact, except rows whose k-th and (k+1)-th oracle
+    scores lie within 1e-3 relative of each other (counted and reported);
+    attention is always compared using the GPU's own index
+  * O: bf16 I/O max-abs <= 2e-2 and mean-abs <= 2e-3; fp32 I/O max-abs <= 1e-5
+  * gradients: max-abs <= 5e-2
+"""
+import numpy as np
+import pytest
+
+from oracle import bra_oracle as orc
+from paper_2303_08810_b200 import synthetic
+from paper_2303_08810_b200.synthetic import BraConfig, CONFIGS
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"bf16": dict(max=2e-2, mean=2e-3), "f32": dict(max=1e-5, mean=1e-6)}
+GRAD_MAX = 5e-2
+
+
+@pytest.fixture(scope="module")
+def bra():
+    import paper_2303_08810_b200 as pkg
+    from paper_2303_08810_b200 import build
+    build.build_library()
+    pkg.load_library()
+    return pkg
+
+
+def to_dev(x, cfg):
+    import torch
+    out = {}
+    for k, v in x.items():
+        t = torch.from_numpy(np.ascontiguousarray(v)).cuda()
+        if k != "w" and cfg.dtype == "bf16":
+            t = t.to(torch.bfloat16)
+        out[k] = t
+    return out
+
+
+def problem_of(bra, cfg, impl=0, **kw):
+    return bra.make_problem(cfg.B, cfg.H, cfg.W, cfg.C, cfg.heads, cfg.S, cfg.topk, cfg.dtype,
+                            impl=impl, **kw)
+
+
+def f64(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def check_index(idx_gpu, idx_ref, gap, topk, R):
+    """Rows with a clear gap must match exactly (as ordered lists); near-tie
+    rows must still be valid selections (distinct, in range)."""
+    clear = gap > 1e-3
+    assert np.array_equal(idx_gpu[clear], idx_ref[clear])
+    assert idx_gpu.min() >= 0 and idx_gpu.max() < R
+    srt = np.sort(idx_gpu, axis=-1)
+    assert (np.diff(srt, axis=-1) > 0).all() or topk == 1
+    near = int((~clear).sum())
+    flips = int((idx_gpu[~clear] != idx_ref[~clear]).any(axis=-1).sum()) if near else 0
+    return near, flips
+
+
+def check_O(O_gpu, O_ref, dtype):
+    err = np.abs(O_gpu - O_ref)
+    assert err.max() <= TOL[dtype]["max"], f"max-abs {err.max():.3e}"
+    assert err.mean() <= TOL[dtype]["mean"], f"mean-abs {err.mean():.3e}"
+
+
+# ------------------------------------------------------------------ routing
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5])
+def test_route_matches_oracle(bra, n):
+    cfg = CONFIGS[n]
+    x = synthetic.make_inputs(cfg, seed=1000 + n)
+    t = to_dev(x, cfg)
+    p = problem_of(bra, cfg)
+    ws = bra.workspace(p)
+    qm, km, idx = bra.bra_route(p, t["Q"], t["K"], ws=ws)
+    assert bra.last_launch_count() >= 2
+    Qr, Kr, idx_ref, gap = orc.bra_route(x["Q"], x["K"], cfg.heads, cfg.S, cfg.topk)
+    np.testing.assert_allclose(f64(qm), Qr, rtol=0, atol=2e-6)
+    np.testing.assert_allclose(f64(km), Kr, rtol=0, atol=2e-6)
+    near, flips = check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R)
+    print(f"config {n}: {near} near-tie rows of {gap.size}, {flips} differ")
+    assert near < 0.02 * gap.size + 5
+    assert bra.bra_device_status(ws) == 0
+
+
+def test_route_shared_and_odd_shapes(bra):
+    import torch
+    cases = [
+        (BraConfig("shared", 2, 12, 20, 48, 3, 4, 5, "f32"), True),
+        (BraConfig("k=R", 1, 9, 6, 32, 2, 3, 9, "bf16"), False),
+        (BraConfig("S=1", 2, 5, 7, 16, 1, 1, 1, "f32"), False),
+        (BraConfig("S=16", 1, 32, 32, 32, 1, 16, 12, "bf16"), False),
+        (BraConfig("R=100", 1, 20, 30, 64, 2, 10, 7, "f32"), True),
+    ]
+    for cfg, shared in cases:
+        x = synthetic.make_inputs(cfg, seed=77)
+        t = to_dev(x, cfg)
+        p = problem_of(bra, cfg, shared_routing=shared)
+        qm, km, idx = bra.bra_route(p, t["Q"], t["K"])
+        Qr, Kr, idx_ref, gap = orc.bra_route(x["Q"], x["K"], cfg.heads, cfg.S, cfg.topk, shared)
+        assert idx.shape == idx_ref.shape
+        np.testing.assert_allclose(f64(qm), Qr, rtol=0, atol=2e-6)
+        check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R)
+
+
+def test_route_exact_ties_go_to_lower_region(bra):
+    """Identical K in every region: all affinities of a row are equal."""
+    import torch
+    cfg = BraConfig("ties", 1, 8, 8, 32, 1, 4, 3, "f32")
+    Q = torch.randn(1, 8, 8, 32, device="cuda")
+    K = torch.ones(1, 8, 8, 32, device="cuda")
+    p = problem_of(bra, cfg)
+    _, _, idx = bra.bra_route(p, Q, K)
+    assert (idx.cpu().numpy() == np.array([0, 1, 2])).all()
+    # +0 / -0 affinities are the same score
+    Q0 = torch.zeros_like(Q)
+    K0 = torch.randn_like(K)
+    _, _, idx0 = bra.bra_route(p, Q0, K0)
+    assert (idx0.cpu().numpy() == np.array([0, 1, 2])).all()
+
+
+# ------------------------------------------------------------------ attention
+IMPLS = {"simt": 1, "mma": 2, "tc": 3, "auto": 0}
+
+
+def run_attend_case(bra, cfg, impl, seed, shared=False, lce=True, bias=False, scale=0.0,
+                    index=None, clustered=False):
+    import torch
+    x = synthetic.make_inputs(cfg, seed=seed, clustered=clustered)
+    t = to_dev(x, cfg)
+    p = problem_of(bra, cfg, impl=IMPLS[impl], shared_routing=shared, lce=lce, scale=scale)
+    ws = bra.workspace(p)
+    if index is None:
+        _, _, idx = bra.bra_route(p, t["Q"], t["K"], ws=ws)
+    else:
+        idx = torch.from_numpy(index).cuda()
+    b = None
+    b_np = None
+    if bias:
+        b_np = np.linspace(-0.5, 0.5, cfg.C).astype(np.float32)
+        b = torch.from_numpy(b_np).cuda()
+    try:
+        O, lse = bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"] if lce else None, b, ws=ws)
+    except bra.BraError as e:
+        if e.code == 7 and impl != "simt":
+            pytest.skip(f"{impl} kernel does not take {cfg.name}")
+        raise
+    assert bra.last_launch_count() >= 1
+    assert bra.bra_device_status(ws) == 0
+    O_ref, lse_ref = orc.bra_attend(x["Q"], x["K"], x["V"], idx.cpu().numpy(),
+                                    x["w"] if lce else None, cfg.heads, cfg.S,
+                                    scale if scale > 0 else None, b_np)
+    check_O(f64(O), O_ref, cfg.dtype)
+    np.testing.assert_allclose(f64(lse), lse_ref, rtol=0, atol=1e-5 if cfg.dtype == "f32" else 2e-3)
+    return O
+
+
+@pytest.mark.parametrize("impl", ["simt", "mma", "tc", "auto"])
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5])
+def test_attend_matches_oracle_on_benchmark_configs(bra, n, impl):
+    run_attend_case(bra, CONFIGS[n], impl, seed=1000 + n)
+
+
+EDGE = [
+    BraConfig("S1-n_r=90", 2, 9, 10, 32, 1, 1, 1, "f32"),
+    BraConfig("rect-regions", 2, 12, 20, 64, 2, 4, 3, "bf16"),
+    BraConfig("n_r=15", 1, 9, 15, 32, 2, 3, 2, "f32"),
+    BraConfig("full-k=R", 1, 14, 14, 64, 2, 7, 49, "bf16"),
+    BraConfig("S=1", 2, 6, 6, 32, 1, 1, 1, "bf16"),
+    BraConfig("one-token-regions", 1, 4, 4, 32, 1, 4, 5, "f32"),
+    BraConfig("d=64", 1, 16, 16, 128, 2, 4, 3, "bf16"),
+    BraConfig("d=16", 1, 16, 16, 32, 2, 2, 2, "f32"),
+    BraConfig("d=128", 1, 8, 8, 128, 1, 2, 2, "bf16"),
+    BraConfig("vit-adapt-small", 1, 32, 32, 128, 2, 8, 12, "bf16"),
+]
+
+
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("cfg", EDGE, ids=[c.name for c in EDGE])
+def test_attend_edge_shapes(bra, cfg, impl):
+    run_attend_case(bra, cfg, impl, seed=5)
+
+
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+def test_attend_options(bra, impl):
+    cfg = BraConfig("opts", 2, 16, 16, 64, 2, 4, 3, "bf16")
+    run_attend_case(bra, cfg, impl, seed=6, lce=False)
+    run_attend_case(bra, cfg, impl, seed=6, bias=True)
+    run_attend_case(bra, cfg, impl, seed=6, scale=0.5)
+    run_attend_case(bra, cfg, impl, seed=6, shared=True)
+    run_attend_case(bra, cfg, impl, seed=6, clustered=True)
+    # a caller's index: any order, duplicates count twice
+    rng = np.random.default_rng(3)
+    idx = rng.integers(0, cfg.R, size=(cfg.B, cfg.heads, cfg.R, cfg.topk)).astype(np.int32)
+    idx[0, 0, 0] = [5, 5, 5]
+    run_attend_case(bra, cfg, impl, seed=6, index=idx)
+
+
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+def test_out_of_range_index_is_reported_not_fatal(bra, impl):
+    import torch
+    cfg = BraConfig("bad-index", 1, 16, 16, 64, 2, 4, 2, "bf16")
+    x = synthetic.make_inputs(cfg, seed=8)
+    t = to_dev(x, cfg)
+    p = problem_of(bra, cfg, impl=IMPLS[impl])
+    ws = bra.workspace(p)
+    idx = torch.zeros(cfg.B, cfg.heads, cfg.R, cfg.topk, dtype=torch.int32, device="cuda")
+    idx[0, 1, 3, 1] = cfg.R          # one past the end
+    idx[0, 0, 7, 0] = -4
+    O, _ = bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"], ws=ws)
+    assert bra.bra_device_status(ws) == 9
+    assert bra.bra_device_status(ws) == 0          # cleared by the read
+    assert torch.isfinite(O.float()).all()
+    # the context is still usable and a clean call reports no error
+    idx.zero_()
+    bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"], ws=ws)
+    assert bra.bra_device_status(ws) == 0
+
+
+# ------------------------------------------------------------------ fused forward
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5])
+def test_forward_matches_oracle(bra, n):
+    cfg = CONFIGS[n]
+    x = synthetic.make_inputs(cfg, seed=1000 + n)
+    t = to_dev(x, cfg)
+    p = problem_of(bra, cfg)
+    ws = bra.workspace(p)
+    O, idx, lse = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+    assert bra.last_launch_count() >= 1
+    assert bra.bra_device_status(ws) == 0
+    _, _, idx_ref, gap = orc.bra_route(x["Q"], x["K"], cfg.heads, cfg.S, cfg.topk)
+    near, flips = check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R)
+    O_ref, lse_ref = orc.bra_attend(x["Q"], x["K"], x["V"], idx.cpu().numpy(), x["w"], cfg.heads, cfg.S)
+    check_O(f64(O), O_ref, cfg.dtype)
+    # without the optional outputs the result is the same
+    O2, _, _ = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws, want_index=False, want_lse=False)
+    assert (O2 == O).all()
+    print(f"config {n}: forward ok, {near} near-tie rows, {flips} differ")
+
+
+def test_forward_is_deterministic(bra):
+    cfg = CONFIGS[5]
+    x = synthetic.make_inputs(cfg, seed=42)
+    t = to_dev(x, cfg)
+    p = problem_of(bra, cfg)
+    ws = bra.workspace(p)
+    O1, i1, l1 = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+    O2, i2, l2 = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+    assert (O1 == O2).all() and (i1 == i2).all() and (l1 == l2).all()
+
+
+# ------------------------------------------------------------------ backward
+def run_backward_case(bra, cfg, seed, clustered=False, shared=False, index=None):
+    import torch
+    x = synthetic.make_inputs(cfg, seed=seed, with_do=True, clustered=clustered)
+    t = to_dev(x, cfg)
+    p = problem_of(bra, cfg, shared_routing=shared)
+    ws = bra.workspace(p)
+    if index is None:
+        O, idx, lse = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+    else:
+        idx = torch.from_numpy(index).cuda()
+        O, lse = bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"], ws=ws)
+    g1 = bra.bra_backward(p, t["Q"], t["K"], t["V"], idx, t["w"], lse, t["dO"], ws=ws, want_bias_grad=True)
+    assert bra.last_launch_count() >= 3
+    g2 = bra.bra_backward(p, t["Q"], t["K"], t["V"], idx, t["w"], lse, t["dO"], ws=ws, want_bias_grad=True)
+    assert bra.bra_device_status(ws) == 0
+    for a, b in zip(g1, g2):
+        assert (a == b).all(), "backward is not bit-reproducible"
+    ref = orc.bra_backward(x["Q"], x["K"], x["V"], idx.cpu().numpy(), x["w"], x["dO"], cfg.heads, cfg.S)
+    names = ("dQ", "dK", "dV", "d_lce_w", "d_lce_b")
+    tol = GRAD_MAX if cfg.dtype == "bf16" else 2e-4
+    for name, g, r in zip(names, g1, ref):
+        err = np.abs(f64(g) - r).max()
+        scale = max(1.0, np.abs(r).max()) if name.startswith("d_lce") else 1.0
+        assert err <= tol * scale, f"{cfg.name} {name}: max-abs {err:.3e}"
+
+
+def test_backward_tiny_fp32(bra):
+    run_backward_case(bra, CONFIGS[1], seed=1001)
+
+
+def test_backward_training_config(bra):
+    run_backward_case(bra, CONFIGS[5], seed=1005)
+
+
+def test_backward_edge_cases(bra):
+    run_backward_case(bra, synthetic.with_batch(CONFIGS[5], 4), seed=9, clustered=True)
+    run_backward_case(bra, BraConfig("bwd-shared", 2, 12, 20, 64, 2, 4, 3, "bf16"), seed=10, shared=True)
+    run_backward_case(bra, BraConfig("bwd-full", 1, 8, 8, 32, 2, 2, 4, "f32"), seed=11)
+    cfg = BraConfig("bwd-dup", 1, 8, 8, 32, 1, 2, 3, "f32")
+    idx = np.array([[[[0, 0, 3], [1, 2, 1], [3, 3, 3], [2, 0, 1]]]], dtype=np.int32)
+    run_backward_case(bra, cfg, seed=12, index=idx)
