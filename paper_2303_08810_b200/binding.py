@@ -68,7 +68,7 @@ def load_library():
     lib.bra_forward.restype = c_int32
     lib.bra_forward.argtypes = [P, v, v, v, v, v, v, v, v, v, c_size_t, v]
     lib.bra_backward.restype = c_int32
-    lib.bra_backward.argtypes = [P] + [v] * 13 + [v, c_size_t, v]
+    lib.bra_backward.argtypes = [P] + [v] * 12 + [v, c_size_t, v]
     lib.bra_device_status.restype = c_int32
     lib.bra_device_status.argtypes = [v, v]
     lib.bra_last_launch_count.restype = c_int32

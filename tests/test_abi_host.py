@@ -110,7 +110,7 @@ def test_null_alignment_workspace_checks(lib):
     assert lib.bra_forward(ref, A, A, None, A, None, A, None, None, A, need, None) == 1
     assert lib.bra_forward(ref, A, A, A, A, None, A, None, None, A, 16, None) == 6
     # backward: lse and dO required
-    args = [A] * 13
+    args = [A] * 12
     bad = list(args); bad[5] = None                                           # lse
     assert lib.bra_backward(ref, *bad, A, need, None) == 1
     bad = list(args); bad[6] = None                                           # dO

@@ -50,17 +50,39 @@ def f64(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-def check_index(idx_gpu, idx_ref, gap, topk, R):
-    """Rows with a clear gap must match exactly (as ordered lists); near-tie
-    rows must still be valid selections (distinct, in range)."""
+def check_index(idx_gpu, idx_ref, gap, topk, R, A=None):
+    """Rows whose k-th and (k+1)-th oracle scores are clearly apart must select
+    exactly the oracle's regions.  The order inside a row must match too, except
+    between neighbours whose oracle scores lie within 1e-3 relative (fp32 and
+    fp64 may rank those either way).  Near-tie rows must still be valid."""
     clear = gap > 1e-3
-    assert np.array_equal(idx_gpu[clear], idx_ref[clear])
+    assert np.array_equal(np.sort(idx_gpu[clear], axis=-1), np.sort(idx_ref[clear], axis=-1))
     assert idx_gpu.min() >= 0 and idx_gpu.max() < R
-    srt = np.sort(idx_gpu, axis=-1)
-    assert (np.diff(srt, axis=-1) > 0).all() or topk == 1
+    if topk > 1:
+        assert (np.diff(np.sort(idx_gpu, axis=-1), axis=-1) > 0).all()
+    order_diff = (idx_gpu != idx_ref).any(axis=-1) & clear
+    if A is not None and order_diff.any():
+        top = np.take_along_axis(A, idx_ref.astype(np.int64), axis=-1)     # descending scores
+        rel = (top[..., :-1] - top[..., 1:]) / np.maximum(
+            np.maximum(np.abs(top[..., :-1]), np.abs(top[..., 1:])), 1e-30)
+        # a row may differ in order only where two neighbouring scores nearly tie
+        assert (rel[order_diff].min(axis=-1) <= 1e-3).all()
+        mism = idx_gpu[order_diff] != idx_ref[order_diff]
+        tie = np.zeros_like(mism)
+        close = rel[order_diff] <= 1e-3
+        tie[:, :-1] |= close
+        tie[:, 1:] |= close
+        assert not (mism & ~tie).any()
+    elif A is None:
+        assert not order_diff.any()
     near = int((~clear).sum())
-    flips = int((idx_gpu[~clear] != idx_ref[~clear]).any(axis=-1).sum()) if near else 0
+    flips = int((np.sort(idx_gpu[~clear], -1) != np.sort(idx_ref[~clear], -1)).any(axis=-1).sum()) if near else 0
     return near, flips
+
+
+def oracle_affinity(x, cfg, shared=False):
+    return orc.region_affinity(orc.region_means(x["Q"], cfg.S), orc.region_means(x["K"], cfg.S),
+                               cfg.heads, shared)
 
 
 def check_O(O_gpu, O_ref, dtype):
@@ -82,7 +104,7 @@ def test_route_matches_oracle(bra, n):
     Qr, Kr, idx_ref, gap = orc.bra_route(x["Q"], x["K"], cfg.heads, cfg.S, cfg.topk)
     np.testing.assert_allclose(f64(qm), Qr, rtol=0, atol=2e-6)
     np.testing.assert_allclose(f64(km), Kr, rtol=0, atol=2e-6)
-    near, flips = check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R)
+    near, flips = check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R, oracle_affinity(x, cfg))
     print(f"config {n}: {near} near-tie rows of {gap.size}, {flips} differ")
     assert near < 0.02 * gap.size + 5
     assert bra.bra_device_status(ws) == 0
@@ -105,7 +127,7 @@ def test_route_shared_and_odd_shapes(bra):
         Qr, Kr, idx_ref, gap = orc.bra_route(x["Q"], x["K"], cfg.heads, cfg.S, cfg.topk, shared)
         assert idx.shape == idx_ref.shape
         np.testing.assert_allclose(f64(qm), Qr, rtol=0, atol=2e-6)
-        check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R)
+        check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R, oracle_affinity(x, cfg, shared))
 
 
 def test_route_exact_ties_go_to_lower_region(bra):
@@ -234,7 +256,7 @@ def test_forward_matches_oracle(bra, n):
     assert bra.last_launch_count() >= 1
     assert bra.bra_device_status(ws) == 0
     _, _, idx_ref, gap = orc.bra_route(x["Q"], x["K"], cfg.heads, cfg.S, cfg.topk)
-    near, flips = check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R)
+    near, flips = check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R, oracle_affinity(x, cfg))
     O_ref, lse_ref = orc.bra_attend(x["Q"], x["K"], x["V"], idx.cpu().numpy(), x["w"], cfg.heads, cfg.S)
     check_O(f64(O), O_ref, cfg.dtype)
     # without the optional outputs the result is the same
