@@ -54,7 +54,8 @@ typedef enum bra_status {
     BRA_ERR_UNSUPPORTED = 7, /* valid problem this build has no kernel for (head dim, lce_ksize, impl) */
     BRA_ERR_CUDA = 8,        /* a CUDA runtime call failed (launch, attribute) */
     BRA_ERR_INDEX = 9,       /* device-detected: routing index entry outside [0, S*S) */
-    BRA_ERR_TIMEOUT = 10     /* device-detected: a bounded wait gave up */
+    BRA_ERR_TIMEOUT = 10,    /* device-detected: a bounded wait gave up */
+    BRA_ERR_STATIC_LIMIT = 11 /* bra_route_static only: B*S*S*C > BRA_ROUTE_STATIC_MAX_MEAN_FLOATS */
 } bra_status;
 
 typedef enum bra_dtype { BRA_F32 = 0, BRA_BF16 = 1 } bra_dtype;
@@ -96,6 +97,40 @@ size_t bra_workspace_bytes(const bra_problem* p);
 bra_status bra_route(const bra_problem* p, const void* Q, const void* K,
                      float* q_mean, float* k_mean, int32_t* index,
                      void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * bra_route for callers that cannot hand over scratch memory.  (The paper has
+ * no counterpart: this is a packaging variant of bra_route, same arithmetic.)
+ *
+ * Who needs it: code that runs where device memory must not be allocated or
+ * sized at call time - a plug-in inside a host application that owns the
+ * memory pool and forbids cudaMalloc, a real-time loop where an allocation's
+ * implicit synchronisation is not acceptable, or a caller that simply has no
+ * allocator to ask for a `ws` buffer.  bra_route needs `ws` (or caller
+ * buffers) for the region means Q^r, K^r between its pooling and its routing
+ * kernel; here those means live in a fixed array inside the library image.
+ *
+ *   Q, K     in   [B,H,W,C] device pointers, as for bra_route
+ *   index    out  int32 [B, heads|1, S*S, topk], as for bra_route (bit-identical result)
+ *
+ * Limits and rules
+ *   - B * S*S * C must not exceed BRA_ROUTE_STATIC_MAX_MEAN_FLOATS, otherwise
+ *     BRA_ERR_STATIC_LIMIT is returned and nothing is launched.  The array
+ *     (2 x that many floats = 4 MiB) is part of the library: every GPU that
+ *     loads it carries the array until the process exits.
+ *   - The call itself allocates nothing on host or device and frees nothing.
+ *   - The first call on each device looks up the array's device address (a
+ *     driver query, no allocation).  Make that first call outside any stream
+ *     capture; later calls on that device only launch kernels.
+ *   - All calls on a device share the one array.  Two calls whose kernels can
+ *     overlap on the GPU (different streams, no dependency) race on it: order
+ *     them.  The array keeps the previous call's means; nothing in it has to
+ *     be zero, because pooling overwrites every element routing then reads.
+ *   - The region means are not returned; use bra_route to get them.
+ */
+#define BRA_ROUTE_STATIC_MAX_MEAN_FLOATS (512 * 1024)
+bra_status bra_route_static(const bra_problem* p, const void* Q, const void* K,
+                            int32_t* index, void* stream);
 
 /*
  * Token-to-token attention over routed regions plus LCE (Eq. 6, Eq. 7, Eq. 1):

@@ -6,7 +6,7 @@ the built library raises.
 """
 from .binding import (  # noqa: F401
     BraProblem, BraError, load_library, make_problem, workspace, workspace_bytes,
-    bra_route, bra_attend, bra_forward, bra_backward, bra_device_status,
+    bra_route, bra_route_static, bra_attend, bra_forward, bra_backward, bra_device_status,
     last_launch_count, status_string, version,
     IMPL_AUTO, IMPL_SIMT, IMPL_MMA, IMPL_TC,
 )

@@ -63,6 +63,8 @@ def load_library():
     lib.bra_workspace_bytes.argtypes = [P]
     lib.bra_route.restype = c_int32
     lib.bra_route.argtypes = [P, v, v, v, v, v, v, c_size_t, v]
+    lib.bra_route_static.restype = c_int32
+    lib.bra_route_static.argtypes = [P, v, v, v, v]
     lib.bra_attend.restype = c_int32
     lib.bra_attend.argtypes = [P, v, v, v, v, v, v, v, v, v, c_size_t, v]
     lib.bra_forward.restype = c_int32
@@ -159,6 +161,27 @@ def bra_route(p, Q, K, q_mean=None, k_mean=None, index=None, ws=None, stream=Non
     _check(lib.bra_route(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(q_mean), _ptr(k_mean), _ptr(index),
                          _ptr(ws), ws.numel(), _stream(stream)), "bra_route")
     return q_mean, k_mean, index
+
+
+ROUTE_STATIC_MAX_MEAN_FLOATS = 512 * 1024
+
+
+def bra_route_static(p, Q, K, index=None, stream=None):
+    """bra_route_static: Q, K -> index, for callers that have no scratch buffer to give.
+
+    The region means stay inside the library (a fixed array of
+    2 x ROUTE_STATIC_MAX_MEAN_FLOATS floats per GPU); the C call allocates
+    nothing.  Pass a preallocated `index` to keep the whole call allocation-free:
+    only when `index` is None does this wrapper ask torch for one.  Calls on
+    one device share the array, so keep them ordered on a stream.
+    """
+    torch = _torch()
+    lib = load_library()
+    if index is None:
+        index = torch.empty(p.B, p.heads_i, p.R, p.topk, dtype=torch.int32, device=Q.device)
+    _check(lib.bra_route_static(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(index), _stream(stream)),
+           "bra_route_static")
+    return index
 
 
 def bra_attend(p, Q, K, V, index, lce_w=None, lce_b=None, O=None, lse=None, ws=None, stream=None,

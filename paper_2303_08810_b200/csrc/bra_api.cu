@@ -57,6 +57,10 @@ static bra_status make_dims(const bra_problem* p, Dims* out) {
     return BRA_OK;
 }
 
+// For translation units that add entry points of their own.
+bra_status check_problem(const bra_problem* p, Dims* out) { return make_dims(p, out); }
+void reset_launch_count() { g_launches = 0; }
+
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 static bra_status check_ws(const Dims& d, const void* ws, size_t ws_bytes, WsLayout* L) {
@@ -236,6 +240,7 @@ const char* bra_status_string(bra_status s) {
         case BRA_ERR_CUDA: return "a CUDA runtime call failed";
         case BRA_ERR_INDEX: return "routing index entry outside [0, S*S) (detected on the device)";
         case BRA_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case BRA_ERR_STATIC_LIMIT: return "problem larger than the built-in scratch of the no-allocation entry point";
     }
     return "unknown status";
 }

@@ -42,6 +42,10 @@ WsLayout ws_layout(const Dims& d);
 
 // Host-side bookkeeping of kernel launches for bra_last_launch_count().
 void count_launch(int n = 1);
+void reset_launch_count();
+
+// Validate a problem statement and fill the derived dimensions.
+bra_status check_problem(const bra_problem* p, Dims* out);
 
 // ---- kernel launchers (each returns the cudaError of its launches) ----------
 cudaError_t launch_pool(const Dims& d, int dtype, const void* Q, const void* K,
