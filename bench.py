@@ -170,7 +170,8 @@ def run_reference(args, cfg):
 def workload_config(cfg, args, extra=None):
     c = {"workload": f"config {args.config}: {cfg.name}", "B": cfg.B, "H": cfg.H, "W": cfg.W,
          "C": cfg.C, "heads": cfg.heads, "S": cfg.S, "topk": cfg.topk, "io_dtype": cfg.dtype,
-         "lce": "5x5 depthwise fused", "parallelism": f"batch-sharded x{args.gpus}, no collective"}
+         "lce": "off" if getattr(args, "no_lce", False) else "5x5 depthwise fused",
+         "parallelism": f"batch-sharded x{args.gpus}, no collective"}
     if extra:
         c.update(extra)
     return c
@@ -186,6 +187,7 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma", "tc"])
     ap.add_argument("--sample-images", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-lce", action="store_true", help="attention term only (lce_ksize = 0)")
     args = ap.parse_args()
 
     from paper_2303_08810_b200 import synthetic
@@ -213,7 +215,8 @@ def main():
     bra.load_library()
 
     impl = {"auto": 0, "simt": 1, "mma": 2, "tc": 3}[args.kernel]
-    p = bra.make_problem(cfg.B, cfg.H, cfg.W, cfg.C, cfg.heads, cfg.S, cfg.topk, cfg.dtype, impl=impl)
+    p = bra.make_problem(cfg.B, cfg.H, cfg.W, cfg.C, cfg.heads, cfg.S, cfg.topk, cfg.dtype, impl=impl,
+                         lce=not args.no_lce)
     tdtype = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     esize = 2 if cfg.dtype == "bf16" else 4
     tensor_bytes = cfg.B * cfg.N * cfg.C * esize

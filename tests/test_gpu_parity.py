@@ -208,9 +208,28 @@ def test_attend_edge_shapes(bra, cfg, impl):
     run_attend_case(bra, cfg, impl, seed=5)
 
 
+# 8 x 8-token regions with head dim 32: the shapes of the persistent tensor-core kernel
+TC_CASES = [
+    BraConfig("tc-k3-two-head-pairs", 2, 32, 32, 128, 4, 4, 3, "bf16"),
+    BraConfig("tc-k16-every-region", 1, 32, 32, 64, 2, 4, 16, "bf16"),
+    BraConfig("tc-several-tiles-per-cta", 5, 56, 56, 64, 2, 7, 2, "bf16"),
+    BraConfig("tc-single-region", 1, 8, 8, 64, 2, 1, 1, "bf16"),
+    BraConfig("tc-k5-S8", 1, 64, 64, 64, 2, 8, 5, "bf16"),
+]
+
+
+@pytest.mark.parametrize("cfg", TC_CASES, ids=[c.name for c in TC_CASES])
+def test_attend_tc_shapes(bra, cfg):
+    run_attend_case(bra, cfg, "tc", seed=21)
+
+
+OPT_CASES = [BraConfig("opts", 2, 16, 16, 64, 2, 4, 3, "bf16"),
+             BraConfig("opts-8x8-regions", 2, 32, 32, 64, 2, 4, 3, "bf16")]
+
+
+@pytest.mark.parametrize("cfg", OPT_CASES, ids=[c.name for c in OPT_CASES])
 @pytest.mark.parametrize("impl", ["simt", "auto"])
-def test_attend_options(bra, impl):
-    cfg = BraConfig("opts", 2, 16, 16, 64, 2, 4, 3, "bf16")
+def test_attend_options(bra, impl, cfg):
     run_attend_case(bra, cfg, impl, seed=6, lce=False)
     run_attend_case(bra, cfg, impl, seed=6, bias=True)
     run_attend_case(bra, cfg, impl, seed=6, scale=0.5)
@@ -223,10 +242,11 @@ def test_attend_options(bra, impl):
     run_attend_case(bra, cfg, impl, seed=6, index=idx)
 
 
+@pytest.mark.parametrize("hw", [16, 32])
 @pytest.mark.parametrize("impl", ["simt", "auto"])
-def test_out_of_range_index_is_reported_not_fatal(bra, impl):
+def test_out_of_range_index_is_reported_not_fatal(bra, impl, hw):
     import torch
-    cfg = BraConfig("bad-index", 1, 16, 16, 64, 2, 4, 2, "bf16")
+    cfg = BraConfig("bad-index", 1, hw, hw, 64, 2, 4, 2, "bf16")
     x = synthetic.make_inputs(cfg, seed=8)
     t = to_dev(x, cfg)
     p = problem_of(bra, cfg, impl=IMPLS[impl])
