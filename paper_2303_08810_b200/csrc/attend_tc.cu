@@ -356,67 +356,47 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
         BRA_TR(n, 5);
 
         // ---- LCE + store ----
-        // One rolled loop over the 12 input rows of the halo: row yy feeds output rows yy - ti
-        // through tap row ti.  Sums p1..p4 hold output rows yy-1..yy-4 with tap rows 0..ti-1
-        // applied; every tap row is applied to every input row without a test (sums of rows
-        // outside the region are formed but never reach a stored row); the sum that took tap
-        // row 4 is complete and leaves as O = O^att + LCE(V).  Loads run one row ahead.
+        // Input row yy of the halo feeds output rows yy - ti through tap row ti.  Fully unrolled:
+        // the 8 x 2 output sums of this thread's channel pair sit in registers under fixed names.
         {
             const uint32_t* halo = reinterpret_cast<const uint32_t*>(smem + OFF_HALO) + lane;
             const uint8_t* stage = smem + OFF_ST;
             uint32_t* out = reinterpret_cast<uint32_t*>(O) +
                             ((((size_t)t.b * dm.H + t.y0) * dm.W + t.x0 + xl0) * dm.C + t.c0) / 2 + lane;
-            float2 p1[2], p2[2], p3[2], p4[2];
+            float2 acc[8][2];
 #pragma unroll
-            for (int xx = 0; xx < 2; ++xx) { p1[xx] = bias2; p2[xx] = bias2; p3[xx] = bias2; p4[xx] = bias2; }
-            uint32_t cur[6];
+            for (int y = 0; y < 8; ++y) { acc[y][0] = bias2; acc[y][1] = bias2; }
+            if (dm.lce) {
 #pragma unroll
-            for (int xx = 0; xx < 6; ++xx) cur[xx] = dm.lce ? halo[(xl0 + xx) * 32] : 0u;
-#pragma unroll 1
-            for (int yy = dm.lce ? 0 : 4; yy < HALO; ++yy) {
-                uint32_t nxt[6];
-                const int yn = yy + 1 < HALO ? yy + 1 : HALO - 1;
+                for (int yy = 0; yy < HALO; ++yy) {
+                    float2 v[6];
 #pragma unroll
-                for (int xx = 0; xx < 6; ++xx) nxt[xx] = dm.lce ? halo[(yn * HALO + xl0 + xx) * 32] : 0u;
-                const int y = yy >= 4 ? yy - 4 : 0;
-                float2 att[2];
+                    for (int xx = 0; xx < 6; ++xx) {
+                        const uint32_t w = halo[(yy * HALO + xl0 + xx) * 32];
+                        v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+                    }
+#pragma unroll
+                    for (int ti = 0; ti < 5; ++ti) {
+                        const int y = yy - ti;
+                        if (y < 0 || y >= 8) continue;
+#pragma unroll
+                        for (int tj = 0; tj < 5; ++tj)
+#pragma unroll
+                            for (int xx = 0; xx < 2; ++xx)
+                                acc[y][xx] = __ffma2_rn(wv[ti * 5 + tj], v[xx + tj], acc[y][xx]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int y = 0; y < 8; ++y)
 #pragma unroll
                 for (int xx = 0; xx < 2; ++xx) {
                     const int tk = y * RS + xl0 + xx;
-                    att[xx] = *reinterpret_cast<const float2*>(
+                    const float2 att = *reinterpret_cast<const float2*>(
                         stage + tk * 256 + (((lane >> 1) ^ (tk & 7)) << 4) + (lane & 1) * 8);
+                    const float2 r = __fadd2_rn(att, acc[y][xx]);
+                    out[((size_t)y * dm.W + xx) * (dm.C / 2)] = pack_bf16(r.x, r.y);
                 }
-                float2 v[6];
-#pragma unroll
-                for (int xx = 0; xx < 6; ++xx)
-                    v[xx] = make_float2(__uint_as_float(cur[xx] << 16), __uint_as_float(cur[xx] & 0xffff0000u));
-                float2 e[2];
-#pragma unroll
-                for (int xx = 0; xx < 2; ++xx) {
-                    e[xx] = p4[xx];
-                    p4[xx] = p3[xx];
-                    p3[xx] = p2[xx];
-                    p2[xx] = p1[xx];
-                    p1[xx] = bias2;
-                }
-#pragma unroll
-                for (int tj = 0; tj < 5; ++tj)
-#pragma unroll
-                    for (int xx = 0; xx < 2; ++xx) {
-                        e[xx] = __ffma2_rn(wv[20 + tj], v[xx + tj], e[xx]);
-                        p4[xx] = __ffma2_rn(wv[15 + tj], v[xx + tj], p4[xx]);
-                        p3[xx] = __ffma2_rn(wv[10 + tj], v[xx + tj], p3[xx]);
-                        p2[xx] = __ffma2_rn(wv[5 + tj], v[xx + tj], p2[xx]);
-                        p1[xx] = __ffma2_rn(wv[tj], v[xx + tj], p1[xx]);
-                    }
-                if (yy >= 4) {
-#pragma unroll
-                    for (int xx = 0; xx < 2; ++xx)
-                        out[((size_t)y * dm.W + xx) * (dm.C / 2)] = pack_bf16(att[xx].x + e[xx].x, att[xx].y + e[xx].y);
-                }
-#pragma unroll
-                for (int xx = 0; xx < 6; ++xx) cur[xx] = nxt[xx];
-            }
         }
         __syncthreads();                    // staging tile (over Q) and halo are free
         BRA_TR(n, 6);
