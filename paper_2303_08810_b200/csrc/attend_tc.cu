@@ -83,17 +83,36 @@ __device__ long long g_trace[32 * 8];
 #endif
 
 struct TileCoord { int b, i, hp, y0, x0, c0; };
-__device__ __forceinline__ TileCoord tile_coord(int T, const Dims& dm) {
-    TileCoord t;
-    const int pairs = dm.heads >> 1;
-    t.hp = T % pairs;
-    t.i = (T / pairs) % dm.R;
-    t.b = T / (pairs * dm.R);
-    t.y0 = (t.i / dm.S) * tc::RS;
-    t.x0 = (t.i % dm.S) * tc::RS;
-    t.c0 = t.hp * 64;
-    return t;
-}
+// Walks tiles T, T + stride, ... (T = (b * R + i) * pairs + hp) with adds and carries only.
+struct TileWalker {
+    int pairs, R, S, inv_s;            // inv_s: i / S == (i * inv_s) >> 20 for i < 4096
+    int d_hp, d_i, d_b;                // stride split into (hp, i, b) digits
+    int hp, i, b;
+    __device__ __forceinline__ void init(int T, int stride, const Dims& dm) {
+        pairs = dm.heads >> 1; R = dm.R; S = dm.S;
+        inv_s = (1 << 20) / S + 1;
+        hp = T % pairs; i = (T / pairs) % R; b = T / (pairs * R);
+        d_hp = stride % pairs; d_i = (stride / pairs) % R; d_b = stride / (pairs * R);
+    }
+    __device__ __forceinline__ void next() {
+        hp += d_hp;
+        int carry = hp >= pairs;
+        hp -= carry ? pairs : 0;
+        i += d_i + carry;
+        carry = i >= R;
+        i -= carry ? R : 0;
+        b += d_b + carry;
+    }
+    __device__ __forceinline__ TileCoord coord() const {
+        TileCoord t;
+        t.b = b; t.i = i; t.hp = hp;
+        const int ry = (i * inv_s) >> 20;
+        t.y0 = ry * tc::RS;
+        t.x0 = (i - ry * S) * tc::RS;
+        t.c0 = hp * 64;
+        return t;
+    }
+};
 
 // K1: topk == 1 (one routed step per tile: no running maximum, no rescaling of O, one K/V buffer).
 template <bool K1>
@@ -124,6 +143,8 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
+    TileWalker walk;
+    walk.init(blockIdx.x, gridDim.x, dm);
 
     // ---- loader mapping: thread copies 16-byte chunk c of the 128-byte channel row (both
     // heads) of token column tx, in token rows lrow..lrow+3 of a region: a warp covers 512
@@ -170,8 +191,9 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     auto load_kv = [&](const TileCoord& t, int2 ent, int buf) {
         int r = lhead ? ent.y : ent.x;
         r = r < 0 ? 0 : r;                  // an invalid entry loads region 0; its P is zero
-        const size_t off = (size_t)t.b * dm.H * row_bytes + (size_t)((r / dm.S) * RS + lrow) * row_bytes +
-                           (size_t)((r % dm.S) * RS + tx) * dm.C * 2 + (size_t)t.c0 * 2 + c * 16;
+        const int ry = (r * walk.inv_s) >> 20, rx = r - ry * dm.S;
+        const size_t off = (size_t)t.b * dm.H * row_bytes + (size_t)(ry * RS + lrow) * row_bytes +
+                           (size_t)(rx * RS + tx) * dm.C * 2 + (size_t)t.c0 * 2 + c * 16;
         const uint32_t kd = sm_base + (buf ? OFF_KV1 : OFF_K) + tile_off;
         const uint32_t vd = sm_base + (buf ? OFF_KV1 + 8192 : OFF_V) + tile_off;
 #pragma unroll
@@ -203,7 +225,7 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
 
     bool ok = true;
     uint32_t n_s = 0, n_o = 0;              // uses of bar_s / bar_o so far (phase parity)
-    TileCoord t = tile_coord(blockIdx.x, dm);
+    TileCoord t = walk.coord();
     int2 ent = read_entries(t, 0);          // entries of the unit whose K/V are being loaded
     if (my_tiles > 0) {
         load_q_halo(t);
@@ -220,7 +242,8 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
             hp_loaded = t.hp;
         }
         const bool has_next = n + 1 < my_tiles;
-        const TileCoord tn = has_next ? tile_coord(blockIdx.x + (n + 1) * gridDim.x, dm) : t;
+        if (has_next) walk.next();
+        const TileCoord tn = has_next ? walk.coord() : t;
 
         float m_run = -INFINITY, l_run = 0.f;
         float o_acc[32];
@@ -338,12 +361,12 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
         // ---- normalise, stage O^att as fp32 [64 tokens][64 ch] (16-byte units xor-swizzled) ----
         {
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            uint8_t* srow = smem + OFF_ST + tq * 256;
+            const uint32_t srow = sm_base + OFF_ST + tq * 256;
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
                 const int chunk = head_half * 8 + q;
-                *reinterpret_cast<float4*>(srow + ((chunk ^ (tq & 7)) << 4)) =
-                    make_float4(o_acc[4 * q] * inv, o_acc[4 * q + 1] * inv, o_acc[4 * q + 2] * inv, o_acc[4 * q + 3] * inv);
+                sts_f32x4(srow + ((chunk ^ (tq & 7)) << 4),
+                          o_acc[4 * q] * inv, o_acc[4 * q + 1] * inv, o_acc[4 * q + 2] * inv, o_acc[4 * q + 3] * inv);
             }
             if (lse)
                 lse[((size_t)t.b * dm.heads + 2 * t.hp + head_half) * dm.N + (size_t)(t.y0 + tq / RS) * dm.W + t.x0 + tq % RS] =
@@ -359,10 +382,11 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
         // Input row yy of the halo feeds output rows yy - ti through tap row ti.  Fully unrolled:
         // the 8 x 2 output sums of this thread's channel pair sit in registers under fixed names.
         {
-            const uint32_t* halo = reinterpret_cast<const uint32_t*>(smem + OFF_HALO) + lane;
-            const uint8_t* stage = smem + OFF_ST;
+            const uint32_t halo = sm_base + OFF_HALO + (xl0 * 32 + lane) * 4;
+            const uint32_t stage = sm_base + OFF_ST + xl0 * 256 + (lane & 1) * 8;
             uint32_t* out = reinterpret_cast<uint32_t*>(O) +
                             ((((size_t)t.b * dm.H + t.y0) * dm.W + t.x0 + xl0) * dm.C + t.c0) / 2 + lane;
+            const size_t out_row = (size_t)dm.W * (dm.C / 2);
             float2 acc[8][2];
 #pragma unroll
             for (int y = 0; y < 8; ++y) { acc[y][0] = bias2; acc[y][1] = bias2; }
@@ -372,7 +396,7 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
                     float2 v[6];
 #pragma unroll
                     for (int xx = 0; xx < 6; ++xx) {
-                        const uint32_t w = halo[(yy * HALO + xl0 + xx) * 32];
+                        const uint32_t w = lds_u32(halo + (yy * HALO + xx) * 128);
                         v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
                     }
 #pragma unroll
@@ -387,16 +411,18 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
                     }
                 }
             }
+            // staging token tk = y * 8 + xl0 + xx: its 16-byte unit index is xor-ed with tk & 7
+            const uint32_t sw0 = (((lane >> 1) ^ (xl0 & 7)) << 4), sw1 = (((lane >> 1) ^ ((xl0 + 1) & 7)) << 4);
 #pragma unroll
-            for (int y = 0; y < 8; ++y)
+            for (int y = 0; y < 8; ++y) {
 #pragma unroll
                 for (int xx = 0; xx < 2; ++xx) {
-                    const int tk = y * RS + xl0 + xx;
-                    const float2 att = *reinterpret_cast<const float2*>(
-                        stage + tk * 256 + (((lane >> 1) ^ (tk & 7)) << 4) + (lane & 1) * 8);
+                    const float2 att = lds_f32x2(stage + (y * RS + xx) * 256 + (xx ? sw1 : sw0));
                     const float2 r = __fadd2_rn(att, acc[y][xx]);
-                    out[((size_t)y * dm.W + xx) * (dm.C / 2)] = pack_bf16(r.x, r.y);
+                    out[xx * (dm.C / 2)] = pack_bf16(r.x, r.y);
                 }
+                out += out_row;
+            }
         }
         __syncthreads();                    // staging tile (over Q) and halo are free
         BRA_TR(n, 6);
