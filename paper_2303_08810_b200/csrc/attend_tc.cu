@@ -6,8 +6,10 @@
 // The two heads are stacked into one 128-row MMA tile:
 //     rows   0..63  = head A queries, rows 64..127 = head B queries
 //     keys   0..63  = head A's routed region, keys 64..127 = head B's
-// S = Q K^T is 128 x 128 of which each row uses its own head's 64 columns; P has
-// zeros in the off-diagonal blocks, so O = P [V_A; V_B] is exact for both heads.
+// S = Q K^T is 128 x 128 of which each row uses its own head's 64 columns.  For O = P V
+// the two heads share the key axis instead: P is 128 x 64 (row r, key j of r's own head)
+// and V is 64 x 64 with key j's row = (head A's channels of token j of A's region | head
+// B's channels of token j of B's region); each row then keeps its own head's 32 columns.
 //
 // Small CTAs (128 threads, ~51 KB of shared memory, 128 TMEM columns), four per SM,
 // each walking its own tiles start to finish; the SM overlaps the CTAs' phases.
@@ -43,14 +45,14 @@ constexpr int RS = 8;            // region side in tokens
 constexpr int HALO = RS + 4;     // 12: region plus the 2-token LCE border
 constexpr int THREADS = 128;
 constexpr int KCAP = 64;         // largest topk
-constexpr int TMEM_COLS = 128;   // S [0,128) fp32; then P [0,64) bf16 pairs + O [64,96)
+constexpr int TMEM_COLS = 128;   // S [0,128) fp32; then P [0,32) bf16 pairs + O [64,128)
 constexpr int TM_O = 64;
 constexpr int HALO_BYTES = HALO * HALO * 128;            // 18432
 // shared memory map (bytes, from a 1024-byte aligned base)
 constexpr int OFF_Q = 0;                                 // [128 rows][64 B]  64B swizzle, K-major
 constexpr int OFF_ST = 0;                                // [64 tokens][64 ch] fp32: over Q, + 8 KB of its own
 constexpr int OFF_K = 16384;                             // [128 keys][64 B]  64B swizzle, K-major (buffer 0)
-constexpr int OFF_V = 24576;                             // [128 keys][64 B]  64B swizzle, MN-major (buffer 0)
+constexpr int OFF_V = 24576;                             // [64 keys][128 B]  128B swizzle, MN-major (buffer 0)
 constexpr int OFF_HALO = 32768;                          // [12][12][64 ch] bf16, linear
 constexpr int OFF_BAR = OFF_HALO + HALO_BYTES;           // 51200: two mbarriers, tmem slot
 constexpr int OFF_KV1 = 52224;                           // topk > 1 only: K buffer 1 (8 KB), V buffer 1 (8 KB)
@@ -153,6 +155,8 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     const int c = tid & 7, tx = (tid >> 3) & 7, lrow = (tid >> 6) * 4;
     const int lhead = c >> 2;
     const uint32_t tile_off = lhead * 4096 + (lrow * 8 + tx) * 64 + (((c & 3) ^ ((tx >> 1) & 3)) << 4);
+    // V: [key][128 B] with both heads side by side, 16-byte chunk index xor-ed with key & 7 (= tx)
+    const uint32_t v_off = (lrow * 8 + tx) * 128 + ((c ^ tx) << 4);
     const size_t row_bytes = (size_t)dm.W * dm.C * 2;
     const uint32_t sm_base = smem_u32(smem);
     const uint8_t* Qb = reinterpret_cast<const uint8_t*>(Qg);
@@ -164,8 +168,8 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     const int tq = tid & 63;                           // query token inside the region
     const uint32_t tg = tmem + ((uint32_t)(warp * 32) << 16);
     const uint32_t s_addr = tg + head_half * 64;       // this row's 64 scores
-    const uint32_t p_addr = tg + head_half * 32;       // this row's 64 probabilities (bf16 pairs)
-    const uint32_t z_addr = tg + (head_half ^ 1) * 32; // the other head's keys: zeros
+    const uint32_t p_addr = tg;                        // this row's 64 probabilities (bf16 pairs)
+    const uint32_t o_addr = tg + TM_O + head_half * 32;   // this row's 32 channels of O
     const float sl2 = dm.scale * 1.4426950408889634f;
     // ---- LCE mapping: warp = 2 columns of the region, lane = channel pair
     const int xl0 = 2 * warp;
@@ -176,7 +180,7 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     int hp_loaded = -1;
 
     constexpr uint32_t IDESC_S = umma_idesc_bf16(128, 128, false, false);
-    constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 32, false, true);
+    constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 64, false, true);
 
     // routing entries (head A, head B) of a unit = (tile, routed step); -1: out of range
     auto read_entries = [&](const TileCoord& t, int m) -> int2 {
@@ -195,11 +199,11 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
         const size_t off = (size_t)t.b * dm.H * row_bytes + (size_t)(ry * RS + lrow) * row_bytes +
                            (size_t)(rx * RS + tx) * dm.C * 2 + (size_t)t.c0 * 2 + c * 16;
         const uint32_t kd = sm_base + (buf ? OFF_KV1 : OFF_K) + tile_off;
-        const uint32_t vd = sm_base + (buf ? OFF_KV1 + 8192 : OFF_V) + tile_off;
+        const uint32_t vd = sm_base + (buf ? OFF_KV1 + 8192 : OFF_V) + v_off;
 #pragma unroll
         for (int i = 0; i < 4; ++i) cp_async_16(kd + i * 512, Kb + off + i * row_bytes, 16);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) cp_async_16(vd + i * 512, Vb + off + i * row_bytes, 16);
+        for (int i = 0; i < 4; ++i) cp_async_16(vd + i * 1024, Vb + off + i * row_bytes, 16);
     };
     auto load_q_halo = [&](const TileCoord& t) {
         const size_t img = (size_t)t.b * dm.H * row_bytes;
@@ -318,23 +322,16 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
                 }
                 tmem_st_32x32b_x8(p_addr + (cc >> 1), pk);
             }
-            {
-                uint32_t z[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) z[q] = 0u;
-#pragma unroll
-                for (int cc = 0; cc < 32; cc += 8) tmem_st_32x32b_x8(z_addr + cc, z);
-            }
             tmem_st_wait();
             tc_fence_before_sync();
             __syncthreads();
             BRA_TR(n, 3);
             if (tid == 0) {
                 tc_fence_after_sync();
-                const uint64_t vd = umma_smem_desc(sm_base + (buf ? OFF_KV1 + 8192 : OFF_V), 16, 512, 4);
-#pragma unroll 1
-                for (int ks = 0; ks < 8; ++ks)         // 128 keys = 8 k-steps of 16
-                    umma_ts(tmem + TM_O, tmem + ks * 8, vd + (uint64_t)(ks * 64), IDESC_O, ks);
+                const uint64_t vd = umma_smem_desc(sm_base + (buf ? OFF_KV1 + 8192 : OFF_V), 16, 1024, 2);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)         // 64 keys = 4 k-steps of 16 (2048 B of V each)
+                    umma_ts(tmem + TM_O, tmem + ks * 8, vd + (uint64_t)(ks * 128), IDESC_O, ks);
                 umma_commit(bar_o);
             }
             ok = mbar_wait(bar_o, n_o & 1, POLL_LIMIT);
@@ -343,7 +340,7 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
             tc_fence_after_sync();
             BRA_TR(n, 4);
             uint32_t oraw[32];
-            tmem_ld_32x32b_x32(tg + TM_O, oraw);
+            tmem_ld_32x32b_x32(o_addr, oraw);
             tmem_ld_wait();
             tc_fence_before_sync();
             if (K1) {
@@ -399,16 +396,17 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
                         const uint32_t w = lds_u32(halo + (yy * HALO + xx) * 128);
                         v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
                     }
+                    // tap column outermost: consecutive FMAs go to different sums
 #pragma unroll
-                    for (int ti = 0; ti < 5; ++ti) {
-                        const int y = yy - ti;
-                        if (y < 0 || y >= 8) continue;
+                    for (int tj = 0; tj < 5; ++tj)
 #pragma unroll
-                        for (int tj = 0; tj < 5; ++tj)
+                        for (int ti = 0; ti < 5; ++ti) {
+                            const int y = yy - ti;
+                            if (y < 0 || y >= 8) continue;
 #pragma unroll
                             for (int xx = 0; xx < 2; ++xx)
                                 acc[y][xx] = __ffma2_rn(wv[ti * 5 + tj], v[xx + tj], acc[y][xx]);
-                    }
+                        }
                 }
             }
             // staging token tk = y * 8 + xl0 + xx: its 16-byte unit index is xor-ed with tk & 7
