@@ -205,6 +205,18 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
 #pragma unroll
         for (int i = 0; i < 4; ++i) cp_async_16(vd + i * 1024, Vb + off + i * row_bytes, 16);
     };
+    // halo chunk i of this thread is token pos = (tid >> 3) + 16 i of the 12 x 12 tile: its byte
+    // offset from the tile's first token, and which map edges would put it outside
+    int32_t h_off[9];
+    uint32_t m_top = 0, m_bot = 0, m_left = 0, m_right = 0;
+#pragma unroll
+    for (int i = 0; i < 9; ++i) {
+        const int pos = (tid >> 3) + 16 * i;
+        const int hy = pos / HALO, hx = pos - hy * HALO;
+        h_off[i] = (hy - 2) * (int32_t)row_bytes + (hx - 2) * dm.C * 2;
+        m_top |= (hy < 2) << i;  m_bot |= (hy >= HALO - 2) << i;
+        m_left |= (hx < 2) << i; m_right |= (hx >= HALO - 2) << i;
+    }
     auto load_q_halo = [&](const TileCoord& t) {
         const size_t img = (size_t)t.b * dm.H * row_bytes;
         const size_t in_row = (size_t)t.c0 * 2 + c * 16;
@@ -215,14 +227,13 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
         if (dm.lce) {
             // 12 x 12 tokens x 128 B around the region, zeros outside the map; 9 chunks per thread
             const uint32_t hd = sm_base + OFF_HALO + tid * 16;
-            int pos = tid >> 3;                       // token of the halo tile, + 16 per step
+            const uint8_t* org = Vb + img + (size_t)t.y0 * row_bytes + (size_t)t.x0 * dm.C * 2 + in_row;
+            const uint32_t outside = (t.y0 == 0 ? m_top : 0u) | (t.y0 + RS == dm.H ? m_bot : 0u) |
+                                     (t.x0 == 0 ? m_left : 0u) | (t.x0 + RS == dm.W ? m_right : 0u);
 #pragma unroll
-            for (int i = 0; i < 9; ++i, pos += 16) {
-                const int hy = pos / HALO, hx = pos - hy * HALO;
-                const int y = t.y0 - 2 + hy, x = t.x0 - 2 + hx;
-                const bool inb = (unsigned)y < (unsigned)dm.H && (unsigned)x < (unsigned)dm.W;
-                const uint8_t* hs = inb ? Vb + img + (size_t)y * row_bytes + (size_t)x * dm.C * 2 + in_row : Vb;
-                cp_async_16(hd + i * 2048, hs, inb ? 16u : 0u);
+            for (int i = 0; i < 9; ++i) {
+                const bool inb = !((outside >> i) & 1u);
+                cp_async_16(hd + i * 2048, inb ? org + h_off[i] : Vb, inb ? 16u : 0u);
             }
         }
     };
@@ -281,7 +292,7 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
             }
             const bool valid = (head_half ? ent_cur.y : ent_cur.x) >= 0;
             BRA_TR(n, 1);
-            ok = mbar_wait(bar_s, n_s & 1, POLL_LIMIT);
+            if (warp == 0) ok = mbar_wait(bar_s, n_s & 1, POLL_LIMIT);   // one warp polls, the rest sleep at the barrier
             ++n_s;
             if (!__syncthreads_and(ok)) { ok = false; break; }
             tc_fence_after_sync();
@@ -334,7 +345,7 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
                     umma_ts(tmem + TM_O, tmem + ks * 8, vd + (uint64_t)(ks * 128), IDESC_O, ks);
                 umma_commit(bar_o);
             }
-            ok = mbar_wait(bar_o, n_o & 1, POLL_LIMIT);
+            if (warp == 0) ok = mbar_wait(bar_o, n_o & 1, POLL_LIMIT);
             ++n_o;
             if (!__syncthreads_and(ok)) { ok = false; break; }
             tc_fence_after_sync();
@@ -452,7 +463,8 @@ static int sm_count() {
 
 bool attend_tc_supported(const Dims& d, int dtype) {
     return dtype == BRA_BF16 && d.d == 32 && d.heads % 2 == 0 && d.hs == tc::RS && d.ws == tc::RS &&
-           d.topk <= tc::KCAP && (long long)d.B * d.R * (d.heads / 2) < (1ll << 30);
+           d.topk <= tc::KCAP && (long long)d.B * d.R * (d.heads / 2) < (1ll << 30) &&
+           (long long)d.W * d.C * 2 * tc::HALO < (1ll << 31) && d.R <= 4096;
 }
 
 cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const void* V,
