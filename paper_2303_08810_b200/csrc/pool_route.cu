@@ -5,41 +5,42 @@
 namespace bra {
 
 // ------------------------------------------------------------------ pooling
-// One CTA reduces one row of regions of one image of one tensor: the hs x W x C
-// strip of tokens it covers is contiguous in memory.  Each thread owns
-// (column x, 16-byte channel vector) pairs, sums the hs rows in registers with
-// independent 16-byte loads, parks the partial sums in shared memory, and the
-// CTA then folds the ws columns of every region.
+// One CTA reduces one region of one image of one tensor.  Thread (x, 16-byte channel
+// vector) sums the hs token rows of its column with up to eight independent 16-byte
+// loads in flight, parks the partial sums in shared memory, and the CTA then folds the
+// ws columns.  Many small CTAs keep a few hundred KB in flight per SM, which is what an
+// HBM-bound scan needs.
 template <typename T> struct Vec;
 template <> struct Vec<float> { static constexpr int n = 4; };
 template <> struct Vec<__nv_bfloat16> { static constexpr int n = 8; };
 
 template <typename T>
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(256)
 pool_kernel(const T* __restrict__ Q, const T* __restrict__ K,
             float* __restrict__ q_mean, float* __restrict__ k_mean, Dims dm) {
     constexpr int VEC = Vec<T>::n;
-    extern __shared__ float part[];   // [W][C]
-    const int ry = blockIdx.x, b = blockIdx.y;
+    extern __shared__ float part[];   // [ws][C]
+    const int r = blockIdx.x, b = blockIdx.y;
+    const int ry = r / dm.S, rx = r - ry * dm.S;
     const T* src = blockIdx.z == 0 ? Q : K;
     float* dst = blockIdx.z == 0 ? q_mean : k_mean;
     const int cvecs = dm.C / VEC;
-    const int items = dm.W * cvecs;
+    const int items = dm.ws * cvecs;                       // one token row of the region
     const size_t row_elems = (size_t)dm.W * dm.C;
-    const T* strip = src + ((size_t)b * dm.H + (size_t)ry * dm.hs) * row_elems;
+    const T* reg = src + ((size_t)b * dm.H + (size_t)ry * dm.hs) * row_elems + (size_t)rx * dm.ws * dm.C;
 
     for (int it = threadIdx.x; it < items; it += blockDim.x) {
         float acc[VEC];
 #pragma unroll
         for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
-        const T* p = strip + (size_t)it * VEC;      // (x, cvec) in row 0 of the strip
+        const T* p = reg + (size_t)it * VEC;               // (x, cvec) in row 0: the region's row is contiguous
         int y = 0;
-        for (; y + 4 <= dm.hs; y += 4) {            // four loads in flight
-            float v[4][VEC];
+        for (; y + 8 <= dm.hs; y += 8) {                    // eight loads in flight
+            float v[8][VEC];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) load_row<VEC>(p + (size_t)(y + u) * row_elems, v[u]);
+            for (int u = 0; u < 8; ++u) load_row<VEC>(p + (size_t)(y + u) * row_elems, v[u]);
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < 8; ++u)
 #pragma unroll
                 for (int i = 0; i < VEC; ++i) acc[i] += v[u][i];
         }
@@ -55,21 +56,20 @@ pool_kernel(const T* __restrict__ Q, const T* __restrict__ K,
     }
     __syncthreads();
     const float inv = 1.0f / (float)dm.n_r;
-    for (int o = threadIdx.x; o < dm.S * dm.C; o += blockDim.x) {
-        const int rx = o / dm.C, c = o - rx * dm.C;
+    for (int c = threadIdx.x; c < dm.C; c += blockDim.x) {
         float s = 0.f;
-        for (int x = 0; x < dm.ws; ++x) s += part[(rx * dm.ws + x) * dm.C + c];
-        dst[((size_t)b * dm.R + ry * dm.S + rx) * dm.C + c] = s * inv;
+        for (int x = 0; x < dm.ws; ++x) s += part[x * dm.C + c];
+        dst[((size_t)b * dm.R + r) * dm.C + c] = s * inv;
     }
 }
 
 cudaError_t launch_pool(const Dims& d, int dtype, const void* Q, const void* K,
                         float* q_mean, float* k_mean, cudaStream_t st) {
     const int vec = dtype == BRA_BF16 ? 8 : 4;
-    int items = d.W * (d.C / vec);
-    int threads = ((items < 1024 ? items : 1024) + 31) / 32 * 32;
-    size_t smem = sizeof(float) * (size_t)d.W * d.C;
-    dim3 grid(d.S, d.B, 2);
+    int items = d.ws * (d.C / vec);
+    int threads = ((items < 256 ? items : 256) + 31) / 32 * 32;
+    size_t smem = sizeof(float) * (size_t)d.ws * d.C;
+    dim3 grid(d.R, d.B, 2);
     cudaError_t e;
     if (dtype == BRA_BF16) {
         if (smem > 48 * 1024 &&
@@ -89,7 +89,7 @@ cudaError_t launch_pool(const Dims& d, int dtype, const void* Q, const void* K,
 }
 
 // ------------------------------------------------------------------ routing
-// One CTA per (image, routing head).  K^r of the head sits in shared memory
+// One CTA per (image, routing head, chunk of 8 affinity rows).  K^r of the head sits in shared memory
 // (row stride odd, so a warp reading one row per lane has no bank conflict).
 // One warp per affinity row: lane l holds the scores of regions l, l+32, ...;
 // the row is sorted by a warp-wide bitonic network on 64-bit keys
@@ -101,36 +101,43 @@ __device__ __forceinline__ uint32_t ordered_bits(float s) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+constexpr int ROWS_PER_CTA = 8;
+
 template <int E>   // E score slots per lane: handles R <= 32 * E
 __global__ void __launch_bounds__(256)
 route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
              int32_t* __restrict__ index, Dims dm) {
-    extern __shared__ float ks[];               // [R][dc + 1]
+    extern __shared__ float4 ks4[];             // [R][dc + 4] floats: rows 16-byte aligned, conflict-free
+    float* ks = reinterpret_cast<float*>(ks4);
     const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
-    const int dc = dm.heads_i == 1 ? dm.C : dm.d;   // channels the affinity sums over
+    const int dc = dm.heads_i == 1 ? dm.C : dm.d;   // channels the affinity sums over (a multiple of 4)
     const int c0 = dm.heads_i == 1 ? 0 : h * dm.d;
-    const int ld = dc + 1;
+    const int ld = dc + 4;
+    const int dc4 = dc >> 2;
     const float* kb = k_mean + (size_t)b * dm.R * dm.C + c0;
-    for (int i = threadIdx.x; i < dm.R * dc; i += blockDim.x) {
-        const int r = i / dc, c = i - r * dc;
-        ks[r * ld + c] = kb[(size_t)r * dm.C + c];
+    for (int i = threadIdx.x; i < dm.R * dc4; i += blockDim.x) {
+        const int r = i / dc4, c4 = i - r * dc4;
+        *reinterpret_cast<float4*>(&ks[r * ld + 4 * c4]) = __ldg(reinterpret_cast<const float4*>(kb + (size_t)r * dm.C) + c4);
     }
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    for (int i = warp; i < dm.R; i += nwarps) {
-        const float* qrow = q_mean + ((size_t)b * dm.R + i) * dm.C + c0;
+    for (int i = blockIdx.y * ROWS_PER_CTA + warp; i < dm.R && i < (int)(blockIdx.y + 1) * ROWS_PER_CTA; i += nwarps) {
+        // lane l scores candidates l, l + 32, ...: channels in increasing order, one fp32 FMA each
+        const float4* qrow = reinterpret_cast<const float4*>(q_mean + ((size_t)b * dm.R + i) * dm.C + c0);
         float acc[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[e] = 0.f;
-        for (int cb = 0; cb < dc; cb += 32) {
-            const float qv = (cb + lane < dc) ? qrow[cb + lane] : 0.f;
-            const int lim = dc - cb < 32 ? dc - cb : 32;
-            for (int c = 0; c < lim; ++c) {
-                const float qc = __shfl_sync(0xffffffffu, qv, c);
+        for (int c4 = 0; c4 < dc4; ++c4) {
+            const float4 q4 = __ldg(qrow + c4);
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const int j = lane + 32 * e;
-                    if (j < dm.R) acc[e] = fmaf(qc, ks[j * ld + cb + c], acc[e]);
+            for (int e = 0; e < E; ++e) {
+                const int j = lane + 32 * e;
+                if (j < dm.R) {
+                    const float4 k4 = *reinterpret_cast<const float4*>(&ks[j * ld + 4 * c4]);
+                    acc[e] = fmaf(q4.x, k4.x, acc[e]);
+                    acc[e] = fmaf(q4.y, k4.y, acc[e]);
+                    acc[e] = fmaf(q4.z, k4.z, acc[e]);
+                    acc[e] = fmaf(q4.w, k4.w, acc[e]);
                 }
             }
         }
@@ -140,6 +147,20 @@ route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
             const int j = lane + 32 * e;
             key[e] = j < dm.R ? ((unsigned long long)ordered_bits(acc[e]) << 32) | (0xffffffffu - (uint32_t)j)
                               : 0ull;
+        }
+        if (dm.topk == 1) {
+            // the row maximum is all that is asked for: one warp reduction
+            unsigned long long best = key[0];
+#pragma unroll
+            for (int e = 1; e < E; ++e) best = key[e] > best ? key[e] : best;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+                best = other > best ? other : best;
+            }
+            if (lane == 0)
+                index[((size_t)b * dm.heads_i + h) * dm.R + i] = (int32_t)(0xffffffffu - (uint32_t)(best & 0xffffffffull));
+            continue;
         }
         // bitonic sort, descending, element id = slot * 32 + lane
 #pragma unroll
@@ -185,11 +206,12 @@ route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
 
 static size_t route_smem(const Dims& d) {
     const int dc = d.heads_i == 1 ? d.C : d.d;
-    return sizeof(float) * (size_t)d.R * (dc + 1);
+    return sizeof(float) * (size_t)d.R * (dc + 4);
 }
 
 bool route_supported(const Dims& d) {
-    return d.R <= 256 && route_smem(d) <= 200 * 1024 && sizeof(float) * (size_t)d.W * d.C <= 200 * 1024;
+    return d.R <= 256 && route_smem(d) <= 200 * 1024 && sizeof(float) * (size_t)d.ws * d.C <= 200 * 1024 &&
+           d.B <= 65535;
 }
 
 template <int E>
@@ -200,7 +222,7 @@ static cudaError_t launch_route_e(const Dims& d, const float* q_mean, const floa
         cudaError_t e = cudaFuncSetAttribute(route_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    route_kernel<E><<<d.B * d.heads_i, 256, smem, st>>>(q_mean, k_mean, index, d);
+    route_kernel<E><<<dim3(d.B * d.heads_i, (d.R + ROWS_PER_CTA - 1) / ROWS_PER_CTA), 256, smem, st>>>(q_mean, k_mean, index, d);
     count_launch();
     return cudaGetLastError();
 }
