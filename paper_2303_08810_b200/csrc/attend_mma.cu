@@ -1,9 +1,404 @@
-// placeholder until the warp-level tensor-core kernel lands
+// Routed token-to-token attention + LCE with warp-level tensor-core MMAs
+// (Eq. 6, Eq. 7 with Eq. 1): head dim 32, bf16, any region shape and any topk.
+//
+// tcgen05 MMAs work on 128-row tiles; a BRA query group is one region's n_r tokens of one
+// head, each group with its own routed keys, so for small regions (n_r = 4 or 16) a 128-row
+// tile would be 8-32x padding.  The warp-level m16n8k16 MMA has the matching granularity:
+// one warp = 16 query rows of one (image, region, head), streaming that group's routed keys
+// in blocks of 64, flash-attention style, with S, P and O in registers.
+//
+// CTA = (image b, query region i, head h, chunk of up to 128 of the region's tokens):
+//   1. all threads: cp.async the Q rows, the V halo of the chunk and, block by block
+//      (double-buffered), the K and V rows of the routed regions: K^g / V^g are never
+//      formed in HBM, the routing index only picks source addresses.  Rows are 64 bytes
+//      (this head's 32 channels) with a 16-byte-chunk xor swizzle for ldmatrix.
+//   2. per warp and key block: S = Q K^T (16 MMAs), online softmax on the fragments
+//      (quad shuffles), O += P V (16 MMAs).
+//   3. normalised O^att to an fp32 staging tile (over the dead K/V buffers).
+//   4. all threads: LCE from the halo tile (thread = channel pair x run of 2 tokens),
+//      + O^att, bf16 store of O.
 #include "bra_internal.h"
+#include "sm100_ptx.cuh"
+
 namespace bra {
-bool attend_mma_supported(const Dims&, int) { return false; }
-cudaError_t launch_attend_mma(const Dims&, const void*, const void*, const void*, const int32_t*,
-                              const float*, const float*, void*, float*, int32_t*, cudaStream_t) {
-    return cudaErrorNotSupported;
+
+using namespace ptx;
+
+namespace wm {
+constexpr int KB = 64;          // keys per block
+constexpr int MAXW = 8;         // warps per CTA at most (128 query rows)
+constexpr int KCAP = 256;       // largest topk
+}  // namespace wm
+
+struct MmaGeom {
+    int nw;            // warps per CTA
+    int chunks;        // token chunks per region
+    int nblocks;       // key blocks per group = ceil(topk * n_r / 64)
+    int stages;        // K/V buffers (1 or 2)
+    int halo_w;        // ws + 4
+    int halo_rows;     // rows of the halo tile (largest chunk) incl. the 4 border rows
+    uint32_t mul_nr, mul_ws, mul_s;   // ceil(2^32 / d) for d = n_r, ws, S
+    int off_q, off_kv, off_flag, off_idx, off_halo, smem_bytes;
+};
+
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, uint32_t d, uint32_t mul) {
+    return d == 1 ? n : __umulhi(n, mul);
 }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t* r) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t* r) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (fp32) += A (bf16, 16x16) * B (bf16, 16x8)
+__device__ __forceinline__ void mma_bf16(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+__global__ void __launch_bounds__(wm::MAXW * 32)
+attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
+                  const __nv_bfloat16* __restrict__ Vg, const int32_t* __restrict__ index,
+                  const float* __restrict__ lce_w, const float* __restrict__ lce_b,
+                  __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
+                  int32_t* __restrict__ status, Dims dm, MmaGeom gm) {
+    using namespace wm;
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t sbase = smem_u32(smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nthreads = gm.nw * 32;
+
+    // ---- which group and chunk ----
+    int bid = blockIdx.x;
+    const int ck = bid % gm.chunks; bid /= gm.chunks;
+    const int h = bid % dm.heads; bid /= dm.heads;
+    const int i = bid % dm.R;
+    const int b = bid / dm.R;
+    const int t0 = ck * gm.nw * 16;                                   // first token of the chunk (raster in region)
+    const int t1 = min(dm.n_r, t0 + gm.nw * 16);
+    const int ry = fdiv(i, dm.S, gm.mul_s), rx = i - ry * dm.S;
+    const int y0 = ry * dm.hs, x0 = rx * dm.ws;                       // region origin in the map
+    const size_t tok_bytes = (size_t)dm.C * 2;
+    const size_t row_bytes = (size_t)dm.W * tok_bytes;
+    const size_t img = (size_t)b * dm.H * row_bytes;
+    const size_t ch_off = (size_t)h * 64;                             // this head's 32 channels
+    const uint8_t* Qb = reinterpret_cast<const uint8_t*>(Qg) + img + ch_off;
+    const uint8_t* Kb = reinterpret_cast<const uint8_t*>(Kg) + img + ch_off;
+    const uint8_t* Vb = reinterpret_cast<const uint8_t*>(Vg) + img + ch_off;
+    const int hi = dm.heads_i == 1 ? 0 : h;
+    const int32_t* irow = index + (((size_t)b * dm.heads_i + hi) * dm.R + i) * dm.topk;
+    const int total_keys = dm.topk * dm.n_r;
+
+    int32_t* s_idx = reinterpret_cast<int32_t*>(smem + gm.off_idx);
+    uint8_t* s_flag = smem + gm.off_flag;                             // [stages][64]: 1 = key counts
+    // ---- routing entries of this group: region origin per slot, -1 if out of range ----
+    for (int m = tid; m < dm.topk; m += nthreads) {
+        int r = __ldg(irow + m);
+        if (r < 0 || r >= dm.R) { record_error(status, BRA_ERR_INDEX, r); r = -1; }
+        s_idx[m] = r;
+    }
+    __syncthreads();
+
+    // ---- loaders ----
+    // one row = one token's 64 bytes of this head = 4 chunks of 16 B, chunk index xor (row >> 1) & 3
+    auto load_row = [&](uint32_t dst_row, int row, const uint8_t* src, bool valid) {
+        const uint32_t sw = (row >> 1) & 3;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            cp_async_16(dst_row + ((q ^ sw) << 4), valid ? src + q * 16 : Kb, valid ? 16u : 0u);
+    };
+    auto load_kv_block = [&](int blk, int stage) {
+        const uint32_t kdst = sbase + gm.off_kv + stage * 8192, vdst = kdst + 4096;
+        for (int key = tid; key < KB; key += nthreads) {
+            const int kk = blk * KB + key;
+            bool valid = kk < total_keys;
+            size_t off = 0;
+            if (valid) {
+                const int m = fdiv(kk, dm.n_r, gm.mul_nr), t = kk - m * dm.n_r;
+                const int r = s_idx[m];
+                valid = r >= 0;
+                if (valid) {
+                    const int qy = fdiv(r, dm.S, gm.mul_s), qx = r - qy * dm.S;
+                    const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
+                    off = (size_t)(qy * dm.hs + ty) * row_bytes + (size_t)(qx * dm.ws + tx) * tok_bytes;
+                }
+            }
+            s_flag[stage * KB + key] = valid ? 1 : 0;
+            load_row(kdst + key * 64, key, Kb + off, valid);
+            load_row(vdst + key * 64, key, Vb + off, valid);
+        }
+    };
+    // Q rows of the chunk (rows beyond the region are zero)
+    for (int row = tid; row < gm.nw * 16; row += nthreads) {
+        const int t = t0 + row;
+        const bool valid = t < dm.n_r;
+        const int ty = fdiv(valid ? t : 0, dm.ws, gm.mul_ws), tx = (valid ? t : 0) - ty * dm.ws;
+        load_row(sbase + gm.off_q + row * 64, row, Qb + (size_t)(y0 + ty) * row_bytes + (size_t)(x0 + tx) * tok_bytes, valid);
+    }
+    // V halo of the chunk's token rows: [rows + 4][ws + 4] tokens x 64 B, zeros outside the map
+    const int cy0 = fdiv(t0, dm.ws, gm.mul_ws);                       // first / last region row of the chunk
+    const int cy1 = fdiv(t1 - 1, dm.ws, gm.mul_ws);
+    const int hrows = cy1 - cy0 + 5;
+    if (dm.lce) {
+        const int cells = hrows * gm.halo_w;
+        for (int cell = tid; cell < cells; cell += nthreads) {
+            const int hy = cell / gm.halo_w, hx = cell - hy * gm.halo_w;
+            const int y = y0 + cy0 + hy - 2, x = x0 + hx - 2;
+            const bool valid = (unsigned)y < (unsigned)dm.H && (unsigned)x < (unsigned)dm.W;
+            const uint8_t* src = Vb + (size_t)(valid ? y : 0) * row_bytes + (size_t)(valid ? x : 0) * tok_bytes;
+            const uint32_t dst = sbase + gm.off_halo + cell * 64;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) cp_async_16(dst + q * 16, valid ? src + q * 16 : Vb, valid ? 16u : 0u);
+        }
+    }
+    load_kv_block(0, 0);
+    cp_async_commit();
+
+    // ---- attention: warp = 16 query rows ----
+    const int g = lane >> 2, tq = lane & 3;                           // fragment row / column pair
+    const float sl2 = dm.scale * 1.4426950408889634f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    float o[4][4];
+#pragma unroll
+    for (int n = 0; n < 4; ++n)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[n][e] = 0.f;
+    uint32_t qa[2][4];
+    const bool lower_only = (t1 - t0) - warp * 16 <= 8;               // rows g + 8 of this warp are padding
+
+    for (int blk = 0; blk < gm.nblocks; ++blk) {
+        const int stage = gm.stages == 2 ? (blk & 1) : 0;
+        if (gm.stages == 2 && blk + 1 < gm.nblocks) {
+            load_kv_block(blk + 1, stage ^ 1);                        // its previous reader finished last iteration
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        if (blk == 0) {
+            // A fragments of Q: ldmatrix x4 per k-step: (rows 0-7, ch lo), (rows 8-15, ch lo), (rows 0-7, ch hi), (rows 8-15, ch hi)
+            const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                const int q = 2 * s + (lane >> 4);
+                ldmatrix_x4(sbase + gm.off_q + row * 64 + ((q ^ ((row >> 1) & 3)) << 4), qa[s]);
+            }
+        }
+        const uint32_t kbase = sbase + gm.off_kv + stage * 8192, vbase = kbase + 4096;
+        // S = Q K^T: 8 key tiles of 8
+        float c[8][4];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
+            uint32_t kb[4];
+            const int key = 8 * j + (lane & 7);
+            const int q = lane >> 3;                                  // channel chunk of this lane's matrix
+            ldmatrix_x4(kbase + key * 64 + ((q ^ ((key >> 1) & 3)) << 4), kb);
+            mma_bf16(c[j], qa[0], kb[0], kb[1]);
+            mma_bf16(c[j], qa[1], kb[2], kb[3]);
+        }
+        // keys that do not count (padding of the last block, out-of-range entries): -inf
+        const uint8_t* fl = s_flag + stage * KB;
+        bool all_valid = true;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uchar2 f = *reinterpret_cast<const uchar2*>(fl + 8 * j + 2 * tq);
+            if (!f.x) { c[j][0] = -INFINITY; c[j][2] = -INFINITY; all_valid = false; }
+            if (!f.y) { c[j][1] = -INFINITY; c[j][3] = -INFINITY; all_valid = false; }
+        }
+        (void)all_valid;
+        // online softmax on rows g (elements 0, 1) and g + 8 (elements 2, 3)
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            mx[0] = fmax3(mx[0], c[j][0], c[j][1]);
+            mx[1] = fmax3(mx[1], c[j][2], c[j][3]);
+        }
+        float corr[2], mneg[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+            const float mnew = fmaxf(m_run[r], mx[r] * sl2);          // sl2 > 0
+            corr[r] = (mnew == -INFINITY) ? 1.f : ex2_approx(m_run[r] - mnew);
+            mneg[r] = (mnew == -INFINITY) ? 0.f : -mnew;
+            m_run[r] = mnew;
+            l_run[r] *= corr[r];
+        }
+#pragma unroll
+        for (int n = 0; n < 4; ++n) { o[n][0] *= corr[0]; o[n][1] *= corr[0]; o[n][2] *= corr[1]; o[n][3] *= corr[1]; }
+        uint32_t pa[4][4];                                            // P as A fragments: 4 k-steps of 16 keys
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float p0 = ex2_approx(fmaf(c[j][0], sl2, mneg[0]));
+            const float p1 = ex2_approx(fmaf(c[j][1], sl2, mneg[0]));
+            float p2 = 0.f, p3 = 0.f;
+            if (!lower_only) {
+                p2 = ex2_approx(fmaf(c[j][2], sl2, mneg[1]));
+                p3 = ex2_approx(fmaf(c[j][3], sl2, mneg[1]));
+            }
+            l_run[0] += p0 + p1;
+            l_run[1] += p2 + p3;
+            pa[j >> 1][(j & 1) * 2] = pack2_bf16(p0, p1);
+            pa[j >> 1][(j & 1) * 2 + 1] = pack2_bf16(p2, p3);
+        }
+        // O += P V: 4 k-steps of 16 keys x 4 channel tiles of 8
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            const int key = 16 * s + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+            for (int np = 0; np < 2; ++np) {
+                uint32_t vb[4];
+                const int q = 2 * np + (lane >> 4);
+                ldmatrix_x4_trans(vbase + key * 64 + ((q ^ ((key >> 1) & 3)) << 4), vb);
+                mma_bf16(o[2 * np], pa[s], vb[0], vb[1]);
+                mma_bf16(o[2 * np + 1], pa[s], vb[2], vb[3]);
+            }
+        }
+        __syncthreads();                                              // this stage may be overwritten
+    }
+
+    // ---- normalise; stage O^att fp32 [token][32 ch] over the K/V buffers; lse ----
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+    }
+    float* stage_o = reinterpret_cast<float*>(smem + gm.off_kv);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int row = warp * 16 + g + 8 * r;
+        const int t = t0 + row;
+        if (t < dm.n_r) {
+            const float inv = l_run[r] > 0.f ? 1.f / l_run[r] : 0.f;
+#pragma unroll
+            for (int n = 0; n < 4; ++n)
+                *reinterpret_cast<float2*>(stage_o + row * 32 + 8 * n + 2 * tq) =
+                    make_float2(o[n][2 * r] * inv, o[n][2 * r + 1] * inv);
+            if (lse && tq == 0) {
+                const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
+                lse[((size_t)b * dm.heads + h) * dm.N + (size_t)(y0 + ty) * dm.W + x0 + tx] =
+                    (m_run[r] + log2f(l_run[r])) * 0.6931471805599453f;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- LCE + store: thread = (channel pair, run of 2 tokens along x when ws is even) ----
+    {
+        const int cp = tid & 15;                                      // channels 2cp, 2cp + 1 of this head
+        const int run = (dm.ws & 1) ? 1 : 2;
+        const int nruns = (t1 - t0) / run;                            // chunk boundaries are multiples of 16 or n_r
+        float2 wv[25];
+        float2 bias2 = make_float2(0.f, 0.f);
+        if (dm.lce) {
+            const float* wp = lce_w + (size_t)(h * 32 + 2 * cp) * 25;
+#pragma unroll
+            for (int q = 0; q < 25; ++q) wv[q] = make_float2(__ldg(wp + q), __ldg(wp + 25 + q));
+            if (lce_b) bias2 = make_float2(__ldg(lce_b + h * 32 + 2 * cp), __ldg(lce_b + h * 32 + 2 * cp + 1));
+        }
+        const uint32_t halo = sbase + gm.off_halo + cp * 4;
+        uint32_t* out = reinterpret_cast<uint32_t*>(O) + (img + ch_off) / 4 + cp;
+        for (int u = tid >> 4; u < nruns; u += nthreads >> 4) {
+            const int t = t0 + u * run;
+            const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
+            float2 acc[2] = {bias2, bias2};
+            if (dm.lce) {
+#pragma unroll
+                for (int ti = 0; ti < 5; ++ti) {
+                    const uint32_t hrow = halo + ((ty - cy0 + ti) * gm.halo_w + tx) * 64;
+                    float2 v[6];
+#pragma unroll
+                    for (int xx = 0; xx < 6; ++xx) {
+                        if (xx < run + 4) {
+                            const uint32_t w = lds_u32(hrow + xx * 64);
+                            v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+                        }
+                    }
+#pragma unroll
+                    for (int tj = 0; tj < 5; ++tj) {
+                        acc[0] = __ffma2_rn(wv[ti * 5 + tj], v[tj], acc[0]);
+                        if (run == 2) acc[1] = __ffma2_rn(wv[ti * 5 + tj], v[tj + 1], acc[1]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                if (e < run) {
+                    const float2 att = *reinterpret_cast<const float2*>(stage_o + (t - t0 + e) * 32 + 2 * cp);
+                    const float2 r2 = __fadd2_rn(att, acc[e]);
+                    out[((size_t)(y0 + ty) * dm.W + x0 + tx + e) * (dm.C / 2)] = pack2_bf16(r2.x, r2.y);
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ host side
+static uint32_t recip32(int d) { return d <= 1 ? 0u : (uint32_t)(((1ull << 32) + (uint64_t)d - 1) / (uint64_t)d); }
+
+static MmaGeom mma_geom(const Dims& d) {
+    MmaGeom g;
+    const int rb = (d.n_r + 15) / 16;
+    g.nw = rb < wm::MAXW ? rb : wm::MAXW;
+    g.chunks = (d.n_r + g.nw * 16 - 1) / (g.nw * 16);
+    g.nblocks = (d.topk * d.n_r + wm::KB - 1) / wm::KB;
+    g.stages = g.nblocks > 1 ? 2 : 1;
+    g.halo_w = d.ws + 4;
+    const int chunk_rows = (g.nw * 16 + d.ws - 1) / d.ws + 1;         // rows a chunk of tokens can touch
+    g.halo_rows = (chunk_rows < d.hs ? chunk_rows : d.hs) + 4;
+    g.mul_nr = recip32(d.n_r); g.mul_ws = recip32(d.ws); g.mul_s = recip32(d.S);
+    int off = 0;
+    g.off_q = off;    off += g.nw * 16 * 64;
+    g.off_kv = off;   off += g.stages * 8192;                         // also the fp32 staging tile: nw * 2 KB
+    g.off_flag = off; off += g.stages * wm::KB;
+    g.off_idx = off;  off += ((d.topk * 4 + 15) / 16) * 16;
+    g.off_halo = off; off += d.lce ? g.halo_rows * g.halo_w * 64 : 0;
+    g.smem_bytes = off;
+    return g;
+}
+
+bool attend_mma_supported(const Dims& d, int dtype) {
+    if (dtype != BRA_BF16 || d.d != 32 || d.topk > wm::KCAP) return false;
+    const MmaGeom g = mma_geom(d);
+    // the staging tile sits over the K/V buffers; chunk boundaries must not split a token run of the LCE
+    if (g.nw * 2048 > g.stages * 8192) return false;
+    if (g.chunks > 1 && ((g.nw * 16) % d.ws) != 0) return false;
+    if ((long long)d.topk * d.n_r * d.n_r >= (1ll << 32) || d.R > 65535 || d.n_r > 65535) return false;
+    return g.smem_bytes <= 200 * 1024 && (long long)d.B * d.R * d.heads * g.chunks < (1ll << 31);
+}
+
+cudaError_t launch_attend_mma(const Dims& d, const void* Q, const void* K, const void* V,
+                              const int32_t* index, const float* lce_w, const float* lce_b,
+                              void* O, float* lse, int32_t* status, cudaStream_t st) {
+    const MmaGeom g = mma_geom(d);
+    static int smem_set = 0;
+    if (g.smem_bytes > 48 * 1024 && g.smem_bytes > smem_set) {
+        cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
+        if (e != cudaSuccess) return e;
+        smem_set = g.smem_bytes;
+    }
+    const unsigned grid = (unsigned)((long long)d.B * d.R * d.heads * g.chunks);
+    attend_mma_kernel<<<grid, g.nw * 32, g.smem_bytes, st>>>(
+        static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
+        static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, g);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace bra

@@ -223,6 +223,37 @@ def test_attend_tc_shapes(bra, cfg):
     run_attend_case(bra, cfg, "tc", seed=21)
 
 
+# head dim 32, bf16, every region shape: the warp-level tensor-core kernel
+MMA_CASES = TC_CASES + [
+    BraConfig("mma-2x2-regions-k16", 2, 14, 14, 256, 8, 7, 16, "bf16"),
+    BraConfig("mma-4x4-regions-k4", 2, 28, 28, 128, 4, 7, 4, "bf16"),
+    BraConfig("mma-16x16-regions-two-chunks", 1, 32, 32, 64, 2, 2, 3, "bf16"),
+    BraConfig("mma-3x5-regions-odd-width", 2, 12, 20, 64, 2, 4, 3, "bf16"),
+    BraConfig("mma-last-block-partial", 1, 14, 14, 64, 2, 7, 49, "bf16"),
+    BraConfig("mma-6x6-region-S1", 2, 6, 6, 32, 1, 1, 1, "bf16"),
+    BraConfig("mma-7x7-regions-k3", 1, 56, 56, 64, 2, 8, 3, "bf16"),
+    BraConfig("mma-one-token-regions", 1, 4, 4, 32, 1, 4, 5, "bf16"),
+    BraConfig("mma-wide-regions-3-chunks", 1, 18, 64, 32, 1, 1, 1, "bf16"),
+]
+
+
+@pytest.mark.parametrize("cfg", MMA_CASES, ids=[c.name for c in MMA_CASES])
+def test_attend_mma_shapes(bra, cfg):
+    run_attend_case(bra, cfg, "mma", seed=22)
+
+
+def test_attend_mma_options(bra):
+    cfg = BraConfig("mma-opts", 2, 16, 16, 64, 2, 4, 3, "bf16")
+    run_attend_case(bra, cfg, "mma", seed=6, lce=False)
+    run_attend_case(bra, cfg, "mma", seed=6, bias=True)
+    run_attend_case(bra, cfg, "mma", seed=6, scale=0.5)
+    run_attend_case(bra, cfg, "mma", seed=6, shared=True)
+    rng = np.random.default_rng(3)
+    idx = rng.integers(0, cfg.R, size=(cfg.B, cfg.heads, cfg.R, cfg.topk)).astype(np.int32)
+    idx[0, 0, 0] = [5, 5, 5]
+    run_attend_case(bra, cfg, "mma", seed=6, index=idx)
+
+
 OPT_CASES = [BraConfig("opts", 2, 16, 16, 64, 2, 4, 3, "bf16"),
              BraConfig("opts-8x8-regions", 2, 32, 32, 64, 2, 4, 3, "bf16")]
 
