@@ -308,11 +308,36 @@ def main():
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    if world > 1:
-        import torch.distributed as dist
-        tt = torch.tensor([ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = tt.tolist()
+    # training configs: the backward pass for the fixed routing index, timed the same way
+    bwd_ms = None
+    if cfg.backward:
+        q, k, v, o = sets[0]
+        lse = torch.empty(cfg.B, cfg.heads, cfg.N, dtype=torch.float32, device=dev)
+        bra.bra_forward(p, q, k, v, w, None, O=o, index=index, lse=lse, ws=ws)
+        g = torch.Generator(device=dev)
+        g.manual_seed(77 + rank)
+        d_o = torch.randn(cfg.B, cfg.H, cfg.W, cfg.C, device=dev, generator=g).to(tdtype)
+        grads = [torch.empty_like(q) for _ in range(3)]
+        d_w = torch.empty(cfg.C, 5, 5, dtype=torch.float32, device=dev)
+        bsteps = max(3, min(args.steps, 20))
+        for _ in range(3):
+            bra.bra_backward(p, q, k, v, index, w, lse, d_o, *grads, d_lce_w=d_w, ws=ws)
+        bwd_launches = bra.last_launch_count()
+        barrier()
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b0.record()
+        for _ in range(bsteps):
+            bra.bra_backward(p, q, k, v, index, w, lse, d_o, *grads, d_lce_w=d_w, ws=ws)
+        b1.record()
+        barrier()
+        bwd_ms = b0.elapsed_time(b1) / bsteps
+        assert bra.bra_device_status(ws) == 0
+
+    from paper_2303_08810_b200 import sharding
+    ms = sharding.max_over_ranks(ms, dev)
+    e2e_ms = sharding.max_over_ranks(e2e_ms, dev)
+    if bwd_ms is not None:
+        bwd_ms = sharding.max_over_ranks(bwd_ms, dev)
     if rank != 0:
         if world > 1:
             import torch.distributed as dist
@@ -349,6 +374,12 @@ def main():
                              "route_us": 1e3 * route_ms, "attend_us": 1e3 * attend_ms,
                              "routed_tflops": flops / (ms / args.steps * 1e-3) / 1e12},
     }
+    if bwd_ms is not None:
+        bwd_bytes = 7 * tensor_bytes + cfg.B * cfg.heads * cfg.N * 4 + index_bytes   # Q,K,V,dO in; dQ,dK,dV out; lse
+        line["backward"] = {"us_per_call": 1e3 * bwd_ms, "gpu_launches_per_call": bwd_launches,
+                            "algorithmic_bytes": bwd_bytes, "achieved_gbs": bwd_bytes / (bwd_ms * 1e-3) / 1e9,
+                            "frac_of_hbm_peak": bwd_bytes / (bwd_ms * 1e-3) / 1e9 / peak,
+                            "note": "fixed routing index; dQ, dK, dV, d_lce_w; L2 state as left by the previous call"}
     traffic_file = os.path.join(ROOT, "profiles", "attend_traffic.json")
     if os.path.exists(traffic_file):
         with open(traffic_file) as f:
