@@ -10,6 +10,7 @@
 //      recomputes P from the saved log-sum-exp, accumulates dK, dV, then adds
 //      the LCE adjoint dV += sum_ij w[c,i,j] dO[y-i+2, x-j+2, c].
 //   4. d_lce_w / d_lce_b: per-CTA partial sums, then a fixed-order final sum.
+// Steps 2 and 3 run on the tensor cores instead (backward_mma.cu) for bf16 with head dim 32.
 #include "bra_internal.h"
 
 namespace bra {
@@ -248,16 +249,22 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-    const long long total = (long long)d.B * d.heads * d.R * d.n_r;
-    const unsigned blocks = (unsigned)((total + 127) / 128);
-    bwd_dq_kernel<T, D><<<blocks, 128, 0, st>>>(q, k, v, index, lse, go, static_cast<T*>(dQ), delta, status, d);
-    count_launch();
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (sizeof(T) == 2 && backward_mma_supported(d, BRA_BF16)) {
+        // head dim 32, bf16: the two tensor-core kernels (dQ + delta, then dK / dV)
+        if ((e = launch_backward_mma(d, Q, K, V, index, inv_off, inv_list, lce_w, lse, dO, dQ, dK, dV,
+                                     delta, status, st)) != cudaSuccess) return e;
+    } else {
+        const long long total = (long long)d.B * d.heads * d.R * d.n_r;
+        const unsigned blocks = (unsigned)((total + 127) / 128);
+        bwd_dq_kernel<T, D><<<blocks, 128, 0, st>>>(q, k, v, index, lse, go, static_cast<T*>(dQ), delta, status, d);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-    bwd_dkv_kernel<T, D><<<blocks, 128, 0, st>>>(q, k, v, inv_off, inv_list, lse, delta, go, lce_w,
-                                                 static_cast<T*>(dK), static_cast<T*>(dV), d);
-    count_launch();
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        bwd_dkv_kernel<T, D><<<blocks, 128, 0, st>>>(q, k, v, inv_off, inv_list, lse, delta, go, lce_w,
+                                                     static_cast<T*>(dK), static_cast<T*>(dV), d);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
 
     if (d.lce || d_lce_b) {
         const long long rows = (long long)d.B * d.H;

@@ -70,6 +70,12 @@ cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const 
                              const int32_t* index, const float* lce_w, const float* lce_b,
                              void* O, float* lse, int32_t* status, cudaStream_t st);
 
+bool backward_mma_supported(const Dims& d, int dtype);
+cudaError_t launch_backward_mma(const Dims& d, const void* Q, const void* K, const void* V,
+                                const int32_t* index, const int32_t* inv_off, const int32_t* inv_list,
+                                const float* lce_w, const float* lse, const void* dO,
+                                void* dQ, void* dK, void* dV, float* delta, int32_t* status, cudaStream_t st);
+
 bool backward_supported(const Dims& d);
 cudaError_t launch_backward(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
                             const int32_t* index, const float* lce_w, const float* lse,

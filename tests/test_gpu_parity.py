@@ -362,6 +362,32 @@ def test_backward_training_config(bra):
     run_backward_case(bra, CONFIGS[5], seed=1005)
 
 
+BWD_MMA_CASES = [
+    BraConfig("bwd-2x2-regions-k16", 2, 14, 14, 256, 8, 7, 16, "bf16"),
+    BraConfig("bwd-8x8-regions-k2", 2, 32, 32, 64, 2, 4, 2, "bf16"),
+    BraConfig("bwd-16x16-regions-multi-block", 1, 32, 32, 64, 2, 2, 3, "bf16"),
+    BraConfig("bwd-last-block-partial", 1, 14, 14, 64, 2, 7, 49, "bf16"),
+    BraConfig("bwd-one-token-regions", 1, 4, 4, 32, 1, 4, 5, "bf16"),
+    BraConfig("bwd-3x5-regions", 2, 12, 20, 64, 2, 4, 3, "bf16"),
+]
+
+
+@pytest.mark.parametrize("cfg", BWD_MMA_CASES, ids=[c.name for c in BWD_MMA_CASES])
+def test_backward_tensor_core_shapes(bra, cfg):
+    run_backward_case(bra, cfg, seed=31)
+
+
+def test_backward_tensor_core_duplicates_and_fan_in(bra):
+    cfg = BraConfig("bwd-dup-bf16", 1, 8, 8, 32, 1, 2, 3, "bf16")
+    idx = np.array([[[[0, 0, 3], [1, 2, 1], [3, 3, 3], [2, 0, 1]]]], dtype=np.int32)
+    run_backward_case(bra, cfg, seed=12, index=idx)
+    # every query region routes to region 0 (largest fan-in) and region 5 is never routed to
+    cfg = BraConfig("bwd-fan-in", 2, 16, 16, 64, 2, 4, 2, "bf16")
+    idx = np.zeros((cfg.B, cfg.heads, cfg.R, cfg.topk), dtype=np.int32)
+    idx[..., 1] = np.arange(cfg.R)[None, None, :] % 5
+    run_backward_case(bra, cfg, seed=13, index=idx)
+
+
 def test_backward_edge_cases(bra):
     run_backward_case(bra, synthetic.with_batch(CONFIGS[5], 4), seed=9, clustered=True)
     run_backward_case(bra, BraConfig("bwd-shared", 2, 12, 20, 64, 2, 4, 3, "bf16"), seed=10, shared=True)
