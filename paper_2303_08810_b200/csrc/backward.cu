@@ -16,31 +16,51 @@
 namespace bra {
 
 // ------------------------------------------------------------ inverse index
-// grid: B * heads_i CTAs; block: R threads rounded up to a warp.
-__global__ void inverse_index_kernel(const int32_t* __restrict__ index, int32_t* __restrict__ inv_off,
-                                     int32_t* __restrict__ inv_list, Dims dm) {
-    extern __shared__ int32_t sm[];   // counts[R + 1]
+// grid: B * heads_i CTAs of 256 threads.  The R * topk entries of the (image, head) are staged
+// in shared memory when they fit.  Warp w takes key regions w, w + 8, ...: it sweeps the entries
+// 32 at a time and finds its region's hits with a ballot, so the list of a key region comes out
+// in entry order (query region, then slot): a fixed order for the dK / dV sums.
+__global__ void __launch_bounds__(256)
+inverse_index_kernel(const int32_t* __restrict__ index, int32_t* __restrict__ inv_off,
+                     int32_t* __restrict__ inv_list, int staged, Dims dm) {
+    extern __shared__ int32_t sm[];   // counts[R + 1], then the staged entries
     const int bh = blockIdx.x;
-    const int32_t* idx = index + (size_t)bh * dm.R * dm.topk;
+    const int32_t* gidx = index + (size_t)bh * dm.R * dm.topk;
     const int entries = dm.R * dm.topk;
-    const int j = threadIdx.x;
-    int count = 0;
-    if (j < dm.R)
-        for (int e = 0; e < entries; ++e) count += (idx[e] == j);
-    if (j < dm.R) sm[j] = count;
+    int32_t* sidx = sm + dm.R + 1;
+    if (staged) {
+        for (int e = threadIdx.x; e < entries; e += blockDim.x) sidx[e] = gidx[e];
+        __syncthreads();
+    }
+    const int32_t* idx = staged ? sidx : gidx;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int j = warp; j < dm.R; j += nwarps) {
+        int count = 0;
+        for (int e0 = 0; e0 < entries; e0 += 32) {
+            const int e = e0 + lane;
+            count += __popc(__ballot_sync(0xffffffffu, e < entries && idx[e] == j));
+        }
+        if (lane == 0) sm[j] = count;
+    }
     __syncthreads();
-    if (j == 0) {
+    if (threadIdx.x == 0) {
         int run = 0;
         for (int r = 0; r < dm.R; ++r) { const int c = sm[r]; sm[r] = run; run += c; }
         sm[dm.R] = run;
     }
     __syncthreads();
     int32_t* off = inv_off + (size_t)bh * (dm.R + 1);
-    if (j <= dm.R) off[j] = sm[j];
-    if (j < dm.R) {
+    for (int j = threadIdx.x; j <= dm.R; j += blockDim.x) off[j] = sm[j];
+    for (int j = warp; j < dm.R; j += nwarps) {
         int32_t* out = inv_list + (size_t)bh * entries + sm[j];
-        for (int e = 0; e < entries; ++e)
-            if (idx[e] == j) *out++ = e / dm.topk;      // the query region of entry e
+        int pos = 0;
+        for (int e0 = 0; e0 < entries; e0 += 32) {
+            const int e = e0 + lane;
+            const bool hit = e < entries && idx[e] == j;
+            const unsigned m = __ballot_sync(0xffffffffu, hit);
+            if (hit) out[pos + __popc(m & ((1u << lane) - 1u))] = e / dm.topk;   // the query region of entry e
+            pos += __popc(m);
+        }
     }
 }
 
@@ -176,53 +196,136 @@ bwd_dkv_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __rest
 }
 
 // ------------------------------------------------------------ d_lce_w, d_lce_b
-// Partial sums: CTA p covers a contiguous range of (image, row) pairs; thread c
-// (one per channel, looped) keeps the 25 tap sums and the bias sum of its channel.
+// Partial sums: CTA p covers a contiguous range of (image, row) pairs.  Thread (channel pair,
+// row slot) keeps the 25 tap sums and the bias sum of its two channels for the rows of its
+// slot; the row slots are then added in a fixed order in shared memory.
+template <typename T> struct Pair;
+template <> struct Pair<float> {
+    static __device__ __forceinline__ float2 load(const float* p) { return __ldg(reinterpret_cast<const float2*>(p)); }
+};
+template <> struct Pair<__nv_bfloat16> {
+    static __device__ __forceinline__ float2 load(const __nv_bfloat16* p) {
+        const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(p));
+        return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    }
+};
+// a channel pair as stored (bf16: one 32-bit word; fp32: two floats) and as two floats
+template <typename T> struct RawPair;
+template <> struct RawPair<float> {
+    typedef float2 type;
+    static __device__ __forceinline__ float2 load(const float* p) { return __ldg(reinterpret_cast<const float2*>(p)); }
+    static __device__ __forceinline__ float2 zero() { return make_float2(0.f, 0.f); }
+    static __device__ __forceinline__ float2 unpack(float2 v) { return v; }
+};
+template <> struct RawPair<__nv_bfloat16> {
+    typedef uint32_t type;
+    static __device__ __forceinline__ uint32_t load(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint32_t*>(p)); }
+    static __device__ __forceinline__ uint32_t zero() { return 0u; }
+    static __device__ __forceinline__ float2 unpack(uint32_t w) {
+        return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    }
+};
+constexpr int DW_SLOTS = 4;     // row slots (blockDim.y)
+constexpr int DW_CP = 64;       // channel pairs per pass (blockDim.x at most)
+
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(DW_CP * DW_SLOTS)
 bwd_dw_partial_kernel(const T* __restrict__ V, const T* __restrict__ dO, float* __restrict__ part,
                       int rows_per_block, Dims dm) {
+    extern __shared__ float2 red[];   // [blockDim.x][26]
     const long long rows = (long long)dm.B * dm.H;
     const long long r0 = (long long)blockIdx.x * rows_per_block;
     const long long r1 = r0 + rows_per_block < rows ? r0 + rows_per_block : rows;
-    for (int c = threadIdx.x; c < dm.C; c += blockDim.x) {
-        float acc[26];
+    const int pairs = dm.C >> 1;
+    for (int cp0 = 0; cp0 < pairs; cp0 += blockDim.x) {
+        const int cp = cp0 + threadIdx.x;
+        const bool active = cp < pairs;
+        float2 acc[26];
 #pragma unroll
-        for (int k = 0; k < 26; ++k) acc[k] = 0.f;
-        for (long long r = r0; r < r1; ++r) {
-            const int b = (int)(r / dm.H), y = (int)(r % dm.H);
-            const size_t img = (size_t)b * dm.N * dm.C;
-            for (int x = 0; x < dm.W; ++x) {
-                const float g = (float)dO[img + ((size_t)y * dm.W + x) * dm.C + c];
-                acc[25] += g;
+        for (int k = 0; k < 26; ++k) acc[k] = make_float2(0.f, 0.f);
+        if (active) {
+            const long long rowp = (long long)dm.W * dm.C;
+            for (long long r = r0 + threadIdx.y; r < r1; r += DW_SLOTS) {
+                const int b = (int)(r / dm.H), y = (int)(r - (long long)b * dm.H);
+                const T* vimg = V + (size_t)b * dm.N * dm.C + 2 * cp;
+                const T* grow = dO + ((size_t)b * dm.N + (size_t)y * dm.W) * dm.C + 2 * cp;
+                const T* vrow[5];
+                bool rv[5];
 #pragma unroll
                 for (int ti = 0; ti < 5; ++ti) {
                     const int yy = y + ti - 2;
-                    if (yy < 0 || yy >= dm.H) continue;
+                    rv[ti] = yy >= 0 && yy < dm.H;
+                    vrow[ti] = vimg + (long long)(rv[ti] ? yy : y) * rowp - 2 * dm.C;
+                }
+                // G positions along x at a time: their 5 x (G + 4) window of V is loaded once (zeros
+                // outside the map), all loads in flight before the first FMA
+                constexpr int G = sizeof(T) == 2 ? 5 : 2;
+                typedef typename RawPair<T>::type raw_t;
+                for (int xb = 0; xb < dm.W; xb += G) {
+                    raw_t win[5][G + 4];
+                    raw_t gr[G];
 #pragma unroll
-                    for (int tj = 0; tj < 5; ++tj) {
-                        const int xx = x + tj - 2;
-                        if (xx < 0 || xx >= dm.W) continue;
-                        acc[ti * 5 + tj] = fmaf(g, (float)V[img + ((size_t)yy * dm.W + xx) * dm.C + c], acc[ti * 5 + tj]);
+                    for (int cc = 0; cc < G + 4; ++cc) {
+                        const bool cv = (unsigned)(xb + cc - 2) < (unsigned)dm.W;
+#pragma unroll
+                        for (int ti = 0; ti < 5; ++ti)
+                            win[ti][cc] = (rv[ti] && cv) ? RawPair<T>::load(vrow[ti] + (size_t)(xb + cc) * dm.C) : RawPair<T>::zero();
+                    }
+#pragma unroll
+                    for (int px = 0; px < G; ++px)
+                        gr[px] = xb + px < dm.W ? RawPair<T>::load(grow + (size_t)(xb + px) * dm.C) : RawPair<T>::zero();
+#pragma unroll
+                    for (int px = 0; px < G; ++px) {
+                        const float2 g = RawPair<T>::unpack(gr[px]);   // zero beyond the row: adds nothing
+                        acc[25] = __fadd2_rn(acc[25], g);
+#pragma unroll
+                        for (int ti = 0; ti < 5; ++ti)
+#pragma unroll
+                            for (int tj = 0; tj < 5; ++tj)
+                                acc[ti * 5 + tj] = __ffma2_rn(g, RawPair<T>::unpack(win[ti][px + tj]), acc[ti * 5 + tj]);
                     }
                 }
             }
         }
-        float* out = part + ((size_t)blockIdx.x * dm.C + c) * 26;
+        // row slots added in the order 0, 1, 2, ...
+        for (int slot = 0; slot < DW_SLOTS; ++slot) {
+            if ((int)threadIdx.y == slot && active) {
 #pragma unroll
-        for (int k = 0; k < 26; ++k) out[k] = acc[k];
+                for (int k = 0; k < 26; ++k)
+                    red[threadIdx.x * 26 + k] = slot == 0 ? acc[k] : __fadd2_rn(red[threadIdx.x * 26 + k], acc[k]);
+            }
+            __syncthreads();
+        }
+        if (threadIdx.y == 0 && active) {
+            float* out = part + ((size_t)blockIdx.x * dm.C + 2 * cp) * 26;
+#pragma unroll
+            for (int k = 0; k < 26; ++k) { out[k] = red[threadIdx.x * 26 + k].x; out[26 + k] = red[threadIdx.x * 26 + k].y; }
+        }
+        __syncthreads();
     }
 }
 
-__global__ void bwd_dw_final_kernel(const float* __restrict__ part, int blocks,
-                                    float* __restrict__ d_lce_w, float* __restrict__ d_lce_b, Dims dm) {
-    const int o = blockIdx.x * blockDim.x + threadIdx.x;   // (channel, slot)
-    if (o >= dm.C * 26) return;
+// Final sum over the partials: 32 outputs per CTA, 8 threads per output each taking every
+// eighth partial in order; the eight slice sums are then added in order.
+__global__ void __launch_bounds__(256)
+bwd_dw_final_kernel(const float* __restrict__ part, int blocks,
+                    float* __restrict__ d_lce_w, float* __restrict__ d_lce_b, Dims dm) {
+    __shared__ float sl[8][32];
+    const int o = blockIdx.x * 32 + threadIdx.x;   // (channel, slot)
+    const int slice = threadIdx.y;
     float s = 0.f;
-    for (int p = 0; p < blocks; ++p) s += part[(size_t)p * dm.C * 26 + o];
-    const int c = o / 26, k = o % 26;
-    if (k < 25) { if (d_lce_w) d_lce_w[c * 25 + k] = s; }
-    else if (d_lce_b) d_lce_b[c] = s;
+    if (o < dm.C * 26)
+        for (int p = slice; p < blocks; p += 8) s += part[(size_t)p * dm.C * 26 + o];
+    sl[slice][threadIdx.x] = s;
+    __syncthreads();
+    if (slice == 0 && o < dm.C * 26) {
+        float t = sl[0][threadIdx.x];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) t += sl[q][threadIdx.x];
+        const int c = o / 26, k = o % 26;
+        if (k < 25) { if (d_lce_w) d_lce_w[c * 25 + k] = t; }
+        else if (d_lce_b) d_lce_b[c] = t;
+    }
 }
 
 bool backward_supported(const Dims& d) {
@@ -244,8 +347,11 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
     const T* v = static_cast<const T*>(V); const T* go = static_cast<const T*>(dO);
     cudaError_t e;
 
-    const int thr = (d.R + 1 + 31) / 32 * 32;
-    inverse_index_kernel<<<d.B * d.heads_i, thr, sizeof(int32_t) * (d.R + 1), st>>>(index, inv_off, inv_list, d);
+    const int thr = 256;
+    const size_t idx_bytes = sizeof(int32_t) * (size_t)d.R * d.topk;
+    const int staged = idx_bytes <= 40 * 1024;
+    inverse_index_kernel<<<d.B * d.heads_i, thr, sizeof(int32_t) * (d.R + 1) + (staged ? idx_bytes : 0), st>>>(
+        index, inv_off, inv_list, staged, d);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
@@ -270,10 +376,11 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
         const long long rows = (long long)d.B * d.H;
         const int rpb = (int)((rows + L.dw_blocks - 1) / L.dw_blocks);
         const int nblk = (int)((rows + rpb - 1) / rpb);
-        bwd_dw_partial_kernel<T><<<nblk, d.C < 256 ? (d.C + 31) / 32 * 32 : 256, 0, st>>>(v, go, part, rpb, d);
+        const int cpx = d.C / 2 < DW_CP ? d.C / 2 : DW_CP;
+        bwd_dw_partial_kernel<T><<<nblk, dim3(cpx, DW_SLOTS), sizeof(float2) * cpx * 26, st>>>(v, go, part, rpb, d);
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        bwd_dw_final_kernel<<<(d.C * 26 + 127) / 128, 128, 0, st>>>(part, nblk, d.lce ? d_lce_w : nullptr, d_lce_b, d);
+        bwd_dw_final_kernel<<<(d.C * 26 + 31) / 32, dim3(32, 8), 0, st>>>(part, nblk, d.lce ? d_lce_w : nullptr, d_lce_b, d);
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
