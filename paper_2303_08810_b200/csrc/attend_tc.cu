@@ -147,6 +147,7 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     const uint32_t tmem = *tmem_slot;
     TileWalker walk;
     walk.init(blockIdx.x, gridDim.x, dm);
+    pdl_wait();          // everything above overlaps the tail of the kernel before (routing, in bra_forward)
 
     // ---- loader mapping: thread copies 16-byte chunk c of the 128-byte channel row (both
     // heads) of token column tx, in token rows lrow..lrow+3 of a region: a warp covers 512
@@ -507,14 +508,17 @@ cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const 
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(Q);
     const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(K);
     const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(V);
+    const bool pdl = take_after_own_kernel();
+    __nv_bfloat16* o = static_cast<__nv_bfloat16*>(O);
+    cudaError_t e;
     if (d.topk == 1)
-        attend_tc_kernel<true><<<grid, tc::THREADS, tc::SMEM_K1, st>>>(
-            q, k, v, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, tiles);
+        e = launch_kernel(attend_tc_kernel<true>, dim3(grid), dim3(tc::THREADS), tc::SMEM_K1, st, pdl,
+                          q, k, v, index, lce_w, lce_b, o, lse, status, d, tiles);
     else
-        attend_tc_kernel<false><<<grid, tc::THREADS, tc::SMEM_KN, st>>>(
-            q, k, v, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, tiles);
+        e = launch_kernel(attend_tc_kernel<false>, dim3(grid), dim3(tc::THREADS), tc::SMEM_KN, st, pdl,
+                          q, k, v, index, lce_w, lce_b, o, lse, status, d, tiles);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace bra

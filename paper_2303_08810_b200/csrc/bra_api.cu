@@ -60,6 +60,9 @@ static bra_status make_dims(const bra_problem* p, Dims* out) {
 // For translation units that add entry points of their own.
 bra_status check_problem(const bra_problem* p, Dims* out) { return make_dims(p, out); }
 void reset_launch_count() { g_launches = 0; }
+static thread_local bool g_after_own = false;
+void hint_after_own_kernel(bool yes) { g_after_own = yes; }
+bool take_after_own_kernel() { const bool v = g_after_own; g_after_own = false; return v; }
 
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -182,8 +185,11 @@ bra_status bra_forward(const bra_problem* p, const void* Q, const void* K, const
     s = run_route(d, p->dtype, Q, K, reinterpret_cast<float*>(w + L.q_mean),
                   reinterpret_cast<float*>(w + L.k_mean), idx, st);
     if (s != BRA_OK) return s;
-    return run_attend(path, d, p->dtype, Q, K, V, idx, lce_w, lce_b, O, lse,
-                      reinterpret_cast<int32_t*>(w + L.status), st);
+    hint_after_own_kernel(true);
+    s = run_attend(path, d, p->dtype, Q, K, V, idx, lce_w, lce_b, O, lse,
+                   reinterpret_cast<int32_t*>(w + L.status), st);
+    hint_after_own_kernel(false);
+    return s;
 }
 
 bra_status bra_backward(const bra_problem* p, const void* Q, const void* K, const void* V,

@@ -43,6 +43,10 @@ WsLayout ws_layout(const Dims& d);
 // Host-side bookkeeping of kernel launches for bra_last_launch_count().
 void count_launch(int n = 1);
 void reset_launch_count();
+// bra_forward tells the attend launcher that the kernel before it in the stream is the
+// library's own routing kernel (so the launch may overlap its tail); read-and-clear.
+void hint_after_own_kernel(bool yes);
+bool take_after_own_kernel();
 
 // Validate a problem statement and fill the derived dimensions.
 bra_status check_problem(const bra_problem* p, Dims* out);
@@ -85,6 +89,25 @@ cudaError_t launch_backward(const Dims& d, int dtype, const void* Q, const void*
 
 // ---- device helpers -----------------------------------------------------------
 #ifdef __CUDACC__
+// Programmatic dependent launch: a kernel launched with launch_kernel(..., after_own_kernel = true)
+// may start while the kernel before it in the stream is still running; pdl_wait() returns once
+// that kernel has completed and its writes are visible (a no-op for an ordinary launch).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 bool after_own_kernel, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_own_kernel ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ void record_error(int32_t* status, int code, int detail) {
     if (atomicCAS(status, 0, code) == 0) status[1] = detail;
 }

@@ -20,6 +20,7 @@ pool_kernel(const T* __restrict__ Q, const T* __restrict__ K,
             float* __restrict__ q_mean, float* __restrict__ k_mean, Dims dm) {
     constexpr int VEC = Vec<T>::n;
     extern __shared__ float part[];   // [ws][C]
+    pdl_launch_dependents();
     const int r = blockIdx.x, b = blockIdx.y;
     const int ry = r / dm.S, rx = r - ry * dm.S;
     const T* src = blockIdx.z == 0 ? Q : K;
@@ -109,6 +110,8 @@ route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
              int32_t* __restrict__ index, Dims dm) {
     extern __shared__ float4 ks4[];             // [R][dc + 4] floats: rows 16-byte aligned, conflict-free
     float* ks = reinterpret_cast<float*>(ks4);
+    pdl_launch_dependents();
+    pdl_wait();                                  // the means come from the kernel before
     const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
     const int dc = dm.heads_i == 1 ? dm.C : dm.d;   // channels the affinity sums over (a multiple of 4)
     const int c0 = dm.heads_i == 1 ? 0 : h * dm.d;
@@ -222,9 +225,10 @@ static cudaError_t launch_route_e(const Dims& d, const float* q_mean, const floa
         cudaError_t e = cudaFuncSetAttribute(route_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    route_kernel<E><<<dim3(d.B * d.heads_i, (d.R + ROWS_PER_CTA - 1) / ROWS_PER_CTA), 256, smem, st>>>(q_mean, k_mean, index, d);
+    cudaError_t e = launch_kernel(route_kernel<E>, dim3(d.B * d.heads_i, (d.R + ROWS_PER_CTA - 1) / ROWS_PER_CTA),
+                                  dim3(256), smem, st, /*after_own_kernel=*/true, q_mean, k_mean, index, d);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_route(const Dims& d, const float* q_mean, const float* k_mean,
