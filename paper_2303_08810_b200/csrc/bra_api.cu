@@ -74,16 +74,18 @@ static bra_status check_ws(const Dims& d, const void* ws, size_t ws_bytes, WsLay
     return BRA_OK;
 }
 
-enum Path { PATH_NONE, PATH_SIMT, PATH_MMA, PATH_TC };
+enum Path { PATH_NONE, PATH_SIMT, PATH_MMA, PATH_TC, PATH_TC_WIDE };
 
 static Path choose_attend(const Dims& d, int dtype, int impl) {
     switch (impl) {
         case BRA_IMPL_SIMT: return attend_simt_supported(d) ? PATH_SIMT : PATH_NONE;
         case BRA_IMPL_MMA:  return attend_mma_supported(d, dtype) ? PATH_MMA : PATH_NONE;
-        case BRA_IMPL_TC:   return attend_tc_supported(d, dtype) ? PATH_TC : PATH_NONE;
+        case BRA_IMPL_TC:   return attend_tc_supported(d, dtype) ? PATH_TC
+                                 : attend_tc_wide_supported(d, dtype) ? PATH_TC_WIDE : PATH_NONE;
         default: break;
     }
     if (attend_tc_supported(d, dtype)) return PATH_TC;
+    if (attend_tc_wide_supported(d, dtype)) return PATH_TC_WIDE;
     if (attend_mma_supported(d, dtype)) return PATH_MMA;
     if (attend_simt_supported(d)) return PATH_SIMT;
     return PATH_NONE;
@@ -105,6 +107,7 @@ static bra_status run_attend(Path path, const Dims& d, int dtype, const void* Q,
         case PATH_SIMT: e = launch_attend_simt(d, dtype, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
         case PATH_MMA:  e = launch_attend_mma(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
         case PATH_TC:   e = launch_attend_tc(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
+        case PATH_TC_WIDE: e = launch_attend_tc_wide(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
         default: return BRA_ERR_UNSUPPORTED;
     }
     return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;

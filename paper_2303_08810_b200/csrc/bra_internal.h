@@ -74,6 +74,11 @@ cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const 
                              const int32_t* index, const float* lce_w, const float* lce_b,
                              void* O, float* lse, int32_t* status, cudaStream_t st);
 
+bool attend_tc_wide_supported(const Dims& d, int dtype);
+cudaError_t launch_attend_tc_wide(const Dims& d, const void* Q, const void* K, const void* V,
+                                  const int32_t* index, const float* lce_w, const float* lce_b,
+                                  void* O, float* lse, int32_t* status, cudaStream_t st);
+
 bool backward_mma_supported(const Dims& d, int dtype);
 cudaError_t launch_backward_mma(const Dims& d, const void* Q, const void* K, const void* V,
                                 const int32_t* index, const int32_t* inv_off, const int32_t* inv_list,

@@ -254,6 +254,31 @@ def test_attend_mma_options(bra):
     run_attend_case(bra, cfg, "mma", seed=6, index=idx)
 
 
+# head dim 32, regions 16 tokens wide and a multiple of 8 high: the tcgen05 kernel for large regions
+TC_WIDE_CASES = [
+    BraConfig("wide-16x16-k4", 2, 32, 32, 64, 2, 2, 4, "bf16"),
+    BraConfig("wide-16x16-k1-three-heads", 1, 32, 32, 96, 3, 2, 1, "bf16"),
+    BraConfig("wide-8x16-regions-k3", 1, 16, 32, 32, 1, 2, 3, "bf16"),
+    BraConfig("wide-24x16-regions", 1, 48, 32, 64, 2, 2, 2, "bf16"),
+    BraConfig("wide-many-tiles", 3, 64, 64, 64, 2, 4, 5, "bf16"),
+]
+
+
+@pytest.mark.parametrize("cfg", TC_WIDE_CASES, ids=[c.name for c in TC_WIDE_CASES])
+def test_attend_tc_wide_shapes(bra, cfg):
+    run_attend_case(bra, cfg, "tc", seed=23)
+
+
+def test_attend_tc_wide_options(bra):
+    cfg = BraConfig("wide-opts", 1, 32, 32, 64, 2, 2, 2, "bf16")
+    run_attend_case(bra, cfg, "tc", seed=6, lce=False)
+    run_attend_case(bra, cfg, "tc", seed=6, bias=True)
+    run_attend_case(bra, cfg, "tc", seed=6, scale=0.5)
+    run_attend_case(bra, cfg, "tc", seed=6, shared=True)
+    idx = np.array([[[[3, 3], [0, 1], [2, 0], [1, 1]]] * 2], dtype=np.int32)
+    run_attend_case(bra, cfg, "tc", seed=6, index=idx)
+
+
 OPT_CASES = [BraConfig("opts", 2, 16, 16, 64, 2, 4, 3, "bf16"),
              BraConfig("opts-8x8-regions", 2, 32, 32, 64, 2, 4, 3, "bf16")]
 
