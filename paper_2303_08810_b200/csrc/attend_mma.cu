@@ -34,6 +34,7 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
     const uint32_t sbase = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nthreads = gm.nw * 32;
+    pdl_wait();          // in bra_forward the launch may overlap the tail of the routing kernel
 
     // ---- which group and chunk ----
     int bid = blockIdx.x;
@@ -324,11 +325,13 @@ cudaError_t launch_attend_mma(const Dims& d, const void* Q, const void* K, const
         smem_set = g.smem_bytes;
     }
     const unsigned grid = (unsigned)((long long)d.B * d.R * d.heads * g.chunks);
-    attend_mma_kernel<<<grid, g.nw * 32, g.smem_bytes, st>>>(
-        static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
-        static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, g);
+    cudaError_t e = launch_kernel(attend_mma_kernel, dim3(grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st,
+                                  take_after_own_kernel(),
+                                  static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
+                                  static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b,
+                                  static_cast<__nv_bfloat16*>(O), lse, status, d, g);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace bra

@@ -15,7 +15,7 @@
 //   one thread    tcgen05.mma O_blk = P V with P read from TMEM; rescaled sum kept in registers
 //   after the last block: normalised O^att to an fp32 staging tile, then LCE (thread =
 //   channel pair x 2 columns x 8 rows, sums in registers) + O^att, one bf16 store of O.
-// 128-thread CTAs, three per SM, each walking its own tiles.  Every wait on an MMA is bounded.
+// 128-thread CTAs, four per SM, each walking its own tiles.  Every wait on an MMA is bounded.
 #include "bra_internal.h"
 #include "sm100_ptx.cuh"
 
@@ -34,11 +34,12 @@ constexpr int TM_O = 64;
 constexpr int HALO_BYTES = HROWS * HCOLS * 64;           // 15360
 // shared memory map (bytes, from a 1024-byte aligned base)
 constexpr int OFF_Q = 0;                                 // [128 rows][64 B]  64B swizzle, K-major
-constexpr int OFF_ST = 0;                                // [128 tokens][32 ch] fp32: over Q, + 8 KB of its own
-constexpr int OFF_KV = 16384;                            // 2 x { K [128 keys][64 B], V [128 keys][64 B] }, 64B swizzle
+constexpr int OFF_ST = 0;                                // [128 tokens][32 ch] fp32: over Q and K buffer 0 (dead by then)
+constexpr int OFF_KV = 8192;                             // 2 x { K [128 keys][64 B], V [128 keys][64 B] }, 64B swizzle
 constexpr int OFF_HALO = OFF_KV + 2 * 16384;             // [12][20][32 ch] bf16, linear
 constexpr int OFF_BAR = OFF_HALO + HALO_BYTES;
-constexpr int SMEM_BYTES = OFF_BAR + 64 + 1024;          // + slack for the manual 1024-byte alignment
+constexpr int ALIGN = 512;                               // the 64-byte swizzle repeats every 512 bytes
+constexpr int SMEM_BYTES = OFF_BAR + 64 + ALIGN;         // + slack for the manual alignment
 constexpr uint32_t POLL_LIMIT = 4000000u;
 }  // namespace tw
 
@@ -52,7 +53,7 @@ __device__ __forceinline__ uint32_t packw(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&h);
 }
 
-__global__ void __launch_bounds__(tw::THREADS, 3)
+__global__ void __launch_bounds__(tw::THREADS, 4)
 attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
                       const __nv_bfloat16* __restrict__ Vg, const int32_t* __restrict__ index,
                       const float* __restrict__ lce_w, const float* __restrict__ lce_b,
@@ -60,7 +61,7 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
                       int32_t* __restrict__ status, Dims dm, int num_tiles) {
     using namespace tw;
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + (ALIGN - 1)) & ~uintptr_t(ALIGN - 1));
     uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem + OFF_BAR);       // S landed in TMEM
     uint64_t* bar_o = bar_s + 1;                                         // O landed in TMEM
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_s + 2);
@@ -338,7 +339,7 @@ cudaError_t launch_attend_tc_wide(const Dims& d, const void* Q, const void* K, c
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
     const int tiles = d.B * d.R * d.heads * (d.hs / tw::RT);
-    const int resident = sms * 3;
+    const int resident = sms * 4;
     const unsigned grid = (unsigned)(tiles < resident ? tiles : resident);
     cudaError_t e = launch_kernel(attend_tc_wide_kernel, dim3(grid), dim3(tw::THREADS), tw::SMEM_BYTES, st,
                                   take_after_own_kernel(),
