@@ -25,7 +25,7 @@ using namespace ptx;
 
 __global__ void __launch_bounds__(wm::MAXW * 32)
 attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
-                  const __nv_bfloat16* __restrict__ Vg, const int32_t* __restrict__ index,
+                  const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
                   const float* __restrict__ lce_w, const float* __restrict__ lce_b,
                   __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
                   int32_t* __restrict__ status, Dims dm, MmaGeom gm) {
@@ -61,7 +61,7 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
     uint8_t* s_flag = smem + gm.off_flag;                             // [stages][64]: 1 = key counts
     // ---- routing entries of this group: region origin per slot, -1 if out of range ----
     for (int m = tid; m < dm.topk; m += nthreads) {
-        int r = __ldg(irow + m);
+        int r = __ldcg(irow + m);   // coherent load: the index may come from the kernel this one overlaps
         if (r < 0 || r >= dm.R) { record_error(status, BRA_ERR_INDEX, r); r = -1; }
         s_idx[m] = r;
     }

@@ -120,7 +120,7 @@ struct TileWalker {
 template <bool K1>
 __global__ void __launch_bounds__(tc::THREADS, K1 ? 4 : 3)
 attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
-                 const __nv_bfloat16* __restrict__ Vg, const int32_t* __restrict__ index,
+                 const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
                  const float* __restrict__ lce_w, const float* __restrict__ lce_b,
                  __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
                  int32_t* __restrict__ status, Dims dm, int num_tiles) {
@@ -183,12 +183,14 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     constexpr uint32_t IDESC_S = umma_idesc_bf16(128, 128, false, false);
     constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 64, false, true);
 
-    // routing entries (head A, head B) of a unit = (tile, routed step); -1: out of range
+    // routing entries (head A, head B) of a unit = (tile, routed step); -1: out of range.  The index may
+    // come from a kernel this one overlaps (programmatic dependent launch): coherent loads after pdl_wait(),
+    // never the read-only path, whose loads the compiler may move above the wait
     auto read_entries = [&](const TileCoord& t, int m) -> int2 {
         const int hA = 2 * t.hp, hB = hA + 1;
         const int hiA = dm.heads_i == 1 ? 0 : hA, hiB = dm.heads_i == 1 ? 0 : hB;
-        int ra = __ldg(index + (((size_t)t.b * dm.heads_i + hiA) * dm.R + t.i) * dm.topk + m);
-        int rb = __ldg(index + (((size_t)t.b * dm.heads_i + hiB) * dm.R + t.i) * dm.topk + m);
+        int ra = __ldcg(index + (((size_t)t.b * dm.heads_i + hiA) * dm.R + t.i) * dm.topk + m);
+        int rb = __ldcg(index + (((size_t)t.b * dm.heads_i + hiB) * dm.R + t.i) * dm.topk + m);
         if (ra < 0 || ra >= dm.R) { record_error(status, BRA_ERR_INDEX, ra); ra = -1; }
         if (rb < 0 || rb >= dm.R) { record_error(status, BRA_ERR_INDEX, rb); rb = -1; }
         return make_int2(ra, rb);

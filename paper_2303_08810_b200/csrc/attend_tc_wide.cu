@@ -55,7 +55,7 @@ __device__ __forceinline__ uint32_t packw(float lo, float hi) {
 
 __global__ void __launch_bounds__(tw::THREADS, 4)
 attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
-                      const __nv_bfloat16* __restrict__ Vg, const int32_t* __restrict__ index,
+                      const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
                       const float* __restrict__ lce_w, const float* __restrict__ lce_b,
                       __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
                       int32_t* __restrict__ status, Dims dm, int num_tiles) {
@@ -134,7 +134,7 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
         }
         // key block u = (routed slot m, row block of that region); entry -1: out of range, its P is zero
         auto load_unit = [&](int u, int buf) -> bool {
-            int r = __ldg(irow + u / RB);
+            int r = __ldcg(irow + u / RB);   // coherent load: the index may come from the kernel this one overlaps
             const bool valid = r >= 0 && r < dm.R;
             if (!valid) { record_error(status, BRA_ERR_INDEX, r); r = 0; }
             const size_t off = (size_t)((r / dm.S) * dm.hs + (u % RB) * RT) * row_bytes + (size_t)((r % dm.S) * WS) * tok_bytes;

@@ -103,13 +103,13 @@ __device__ __forceinline__ uint32_t ordered_bits(float s) {
 }
 
 constexpr int ROWS_PER_CTA = 8;
+constexpr int SELECT_MAX_K = 8;             // up to here k rounds of a warp maximum beat the full sort
 
 template <int E>   // E score slots per lane: handles R <= 32 * E
 __global__ void __launch_bounds__(256)
-route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
-             int32_t* __restrict__ index, Dims dm) {
-    extern __shared__ float4 ks4[];             // [R][dc + 4] floats: rows 16-byte aligned, conflict-free
-    float* ks = reinterpret_cast<float*>(ks4);
+route_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ index, Dims dm) {
+    extern __shared__ float4 ks4[];             // [R][dc + 4] floats: rows 16-byte aligned, conflict-free;
+    float* ks = reinterpret_cast<float*>(ks4);  // then this CTA's rows of Q^r, [8][dc]
     pdl_launch_dependents();
     pdl_wait();                                  // the means come from the kernel before
     const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
@@ -120,18 +120,26 @@ route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
     const float* kb = k_mean + (size_t)b * dm.R * dm.C + c0;
     for (int i = threadIdx.x; i < dm.R * dc4; i += blockDim.x) {
         const int r = i / dc4, c4 = i - r * dc4;
-        *reinterpret_cast<float4*>(&ks[r * ld + 4 * c4]) = __ldg(reinterpret_cast<const float4*>(kb + (size_t)r * dm.C) + c4);
+        *reinterpret_cast<float4*>(&ks[r * ld + 4 * c4]) = __ldcg(reinterpret_cast<const float4*>(kb + (size_t)r * dm.C) + c4);
+    }
+    float* qs = ks + (size_t)dm.R * ld;
+    const int row0 = blockIdx.y * ROWS_PER_CTA;
+    const float* qb = q_mean + ((size_t)b * dm.R + row0) * dm.C + c0;
+    for (int i = threadIdx.x; i < ROWS_PER_CTA * dc4; i += blockDim.x) {
+        const int r = i / dc4, c4 = i - r * dc4;
+        if (row0 + r < dm.R)
+            *reinterpret_cast<float4*>(&qs[r * dc + 4 * c4]) = __ldcg(reinterpret_cast<const float4*>(qb + (size_t)r * dm.C) + c4);
     }
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     for (int i = blockIdx.y * ROWS_PER_CTA + warp; i < dm.R && i < (int)(blockIdx.y + 1) * ROWS_PER_CTA; i += nwarps) {
         // lane l scores candidates l, l + 32, ...: channels in increasing order, one fp32 FMA each
-        const float4* qrow = reinterpret_cast<const float4*>(q_mean + ((size_t)b * dm.R + i) * dm.C + c0);
+        const float4* qrow = reinterpret_cast<const float4*>(qs + (i - row0) * dc);
         float acc[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[e] = 0.f;
         for (int c4 = 0; c4 < dc4; ++c4) {
-            const float4 q4 = __ldg(qrow + c4);
+            const float4 q4 = qrow[c4];
 #pragma unroll
             for (int e = 0; e < E; ++e) {
                 const int j = lane + 32 * e;
@@ -163,6 +171,25 @@ route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
             }
             if (lane == 0)
                 index[((size_t)b * dm.heads_i + h) * dm.R + i] = (int32_t)(0xffffffffu - (uint32_t)(best & 0xffffffffull));
+            continue;
+        }
+        int32_t* out = index + (((size_t)b * dm.heads_i + h) * dm.R + i) * dm.topk;
+        if (dm.topk <= SELECT_MAX_K) {
+            // a few winners: one warp-wide maximum per rank, the winner's key cleared for the next round
+            for (int m = 0; m < dm.topk; ++m) {
+                unsigned long long best = key[0];
+#pragma unroll
+                for (int e = 1; e < E; ++e) best = key[e] > best ? key[e] : best;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+                    best = other > best ? other : best;
+                }
+#pragma unroll
+                for (int e = 0; e < E; ++e)
+                    if (key[e] == best) key[e] = 0ull;       // keys are distinct: they carry the region number
+                if (lane == 0) out[m] = (int32_t)(0xffffffffu - (uint32_t)(best & 0xffffffffull));
+            }
             continue;
         }
         // bitonic sort, descending, element id = slot * 32 + lane
@@ -198,7 +225,6 @@ route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
                 }
             }
         }
-        int32_t* out = index + (((size_t)b * dm.heads_i + h) * dm.R + i) * dm.topk;
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             const int rank = e * 32 + lane;
@@ -209,7 +235,7 @@ route_kernel(const float* __restrict__ q_mean, const float* __restrict__ k_mean,
 
 static size_t route_smem(const Dims& d) {
     const int dc = d.heads_i == 1 ? d.C : d.d;
-    return sizeof(float) * (size_t)d.R * (dc + 4);
+    return sizeof(float) * ((size_t)d.R * (dc + 4) + (size_t)ROWS_PER_CTA * dc);
 }
 
 bool route_supported(const Dims& d) {

@@ -352,6 +352,32 @@ def test_forward_is_deterministic(bra):
     assert (O1 == O2).all() and (i1 == i2).all() and (l1 == l2).all()
 
 
+@pytest.mark.parametrize("n", [2, 3, 4, 5])
+def test_forward_orders_attention_after_routing(bra, n):
+    """The library's kernels overlap (programmatic dependent launch): attention must still see the
+    index the routing step of the SAME call wrote.  Each call starts from an index buffer full of
+    out-of-range entries and another pair of Q, K, so a kernel that read the buffer too early would
+    either report a bad index or attend to the regions of the call before."""
+    import torch
+    cfg = CONFIGS[n]
+    p = problem_of(bra, cfg)
+    ws = bra.workspace(p)
+    sets = [to_dev(synthetic.make_inputs(cfg, seed=77 + s), cfg) for s in range(2)]
+    want = []
+    for t in sets:
+        _, _, idx = bra.bra_route(p, t["Q"], t["K"], ws=ws)
+        O, _ = bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"], ws=ws)
+        want.append((idx.clone(), O.clone()))
+    assert bra.bra_device_status(ws) == 0
+    idx = torch.empty_like(want[0][0])
+    for it in range(6):
+        t, (idx_ref, O_ref) = sets[it % 2], want[it % 2]
+        idx.fill_(-7)
+        O, idx, _ = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], index=idx, ws=ws)
+        assert bra.bra_device_status(ws) == 0, f"call {it}"
+        assert (idx == idx_ref).all() and (O == O_ref).all(), f"call {it}"
+
+
 # ------------------------------------------------------------------ backward
 def run_backward_case(bra, cfg, seed, clustered=False, shared=False, index=None):
     import torch
