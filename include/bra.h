@@ -65,7 +65,9 @@ typedef enum bra_impl {
     BRA_IMPL_AUTO = 0,  /* fastest kernel that supports the problem */
     BRA_IMPL_SIMT = 1,  /* fp32 CUDA-core kernel: any dtype, any shape with C/heads <= 128 */
     BRA_IMPL_MMA = 2,   /* bf16 warp-level tensor-core kernel (C/heads == 32) */
-    BRA_IMPL_TC = 3     /* bf16 tcgen05/TMEM kernels (C/heads == 32; regions of 8 x 8 tokens, or 16 wide and a multiple of 8 high) */
+    BRA_IMPL_TC = 3,    /* bf16 tcgen05/TMEM kernels (C/heads == 32; regions of 8 x 8 tokens, or 16 wide and a multiple of 8 high) */
+    BRA_IMPL_IMG = 4    /* bf16 warp-level tensor-core kernel with a whole (image, head) of K and V resident in
+                           shared memory (C/heads == 32, H*W <= ~1500 tokens): small maps, small regions */
 } bra_impl;
 
 /* Problem statement in the notation of Algorithm 1 (H, W, C, S, k) plus batch and heads. */

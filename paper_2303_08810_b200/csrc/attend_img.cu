@@ -1,0 +1,454 @@
+// Routed token-to-token attention + LCE for small feature maps, with the keys and values
+// of a whole (image, head) resident in shared memory (Eq. 6, Eq. 7 with Eq. 1).
+//
+// Late stages of the network have few tokens per image (14 x 14 or 28 x 28) and small regions
+// (2 x 2 or 4 x 4 tokens) with many routed regions per query.  A kernel that copies the routed
+// K / V tiles and a V halo per (region, head) group then moves every key 16 times and every
+// value ~20 times from L2.  Here one CTA owns (image b, head h):
+//   1. all threads: cp.async the head's 64-byte slice of every K and V token of the image into
+//      shared memory, once (N x 128 bytes; 16-byte chunks xor-swizzled for ldmatrix), plus the
+//      head's routing index rows and its LCE weights.  K^g / V^g are never formed anywhere: the
+//      "gather" of Eq. 6 is the row addresses that ldmatrix is given.
+//   2. each warp, on its own, takes units of 16 query tokens of one region: Q fragments straight
+//      from global memory, then per block of 64 routed keys S = Q K^T (m16n8k16 MMAs whose B rows
+//      are picked by the routing index), online softmax on the fragments, O += P V.
+//   3. the warp parks its normalised O^att tile (fp32, warp-private), adds the 5 x 5 depthwise
+//      correlation of V read from the resident V slice (zero outside the map) and stores bf16.
+// No CTA-wide barrier after the set-up: the warps never wait for one another.
+#include "mma_common.cuh"
+
+namespace bra {
+
+using namespace ptx;
+
+namespace img {
+constexpr int KB = 64;            // keys per block
+constexpr int MAX_WARPS = 8;
+constexpr int MAX_ENTRIES = 8192; // routing entries of one (image, head): R * topk
+}  // namespace img
+
+struct ImgGeom {
+    int nw;                 // warps per CTA
+    int tpr;                // 16-row query tiles per region
+    int units;              // R * tpr
+    int nblocks;            // key blocks per unit = ceil(topk * n_r / 64)
+    uint32_t mul_nr, mul_ws, mul_s, mul_tpr;
+    int off_k, off_v, off_idx, off_w, off_st, smem_bytes;
+};
+
+__device__ __forceinline__ uint32_t ldg_u32(const uint8_t* p) {
+    return __ldg(reinterpret_cast<const uint32_t*>(p));
+}
+
+
+// 5 x 5 depthwise correlation (LCE) of the resident V slice for a block of BR rows x WS columns of
+// tokens whose top-left token is (y, x) of the map, for one channel pair: sums added into acc.
+// WS and x are even, so the tokens of a window row pair up on one swizzle phase: one address per
+// pair of loads.  BORDER: the 2-token frame of the block may leave the map (zeros there).
+template <int WS, int BR, bool BORDER>
+__device__ __forceinline__ void lce_block(uint32_t vbase, int y, int x, int H, int W, int cq, uint32_t vcol,
+                                          const float2* wv, float2 (*acc)[WS]) {
+    constexpr int WW = WS + 4;
+#pragma unroll
+    for (int yy = 0; yy < BR + 4; ++yy) {
+        const int iy = y + yy - 2;
+        const bool row_ok = !BORDER || (unsigned)iy < (unsigned)H;
+        const int rt = iy * W + x - 2;                       // token id of the window row's first column
+        float2 v[WW];
+#pragma unroll
+        for (int j = 0; j < WW / 2; ++j) {
+            const int tok = rt + 2 * j;                      // even: tok and tok + 1 share (tok >> 1) & 3
+            const uint32_t a = vbase + tok * 64 + ((cq ^ ((tok >> 1) & 3)) << 4) + vcol;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int ix = x + 2 * j + e - 2;
+                uint32_t w = 0u;
+                if (row_ok && (!BORDER || (unsigned)ix < (unsigned)W)) w = lds_u32(a + e * 64);
+                v[2 * j + e] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+            }
+        }
+#pragma unroll
+        for (int tj = 0; tj < 5; ++tj)
+#pragma unroll
+            for (int ti = 0; ti < 5; ++ti) {
+                const int r = yy - ti;
+                if (r < 0 || r >= BR) continue;
+#pragma unroll
+                for (int c = 0; c < WS; ++c) acc[r][c] = __ffma2_rn(wv[ti * 5 + tj], v[c + tj], acc[r][c]);
+            }
+    }
+}
+
+// One lane's share of a unit whose 16 (or 4) tokens form full region rows: BR rows x WS columns from
+// row r0 of the tile; adds the parked O^att and stores bf16.
+template <int WS, int BR>
+__device__ __forceinline__ void lce_store_block(uint32_t vbase, const float* stage_o, uint32_t* outb, int r0,
+                                                int y0, int x0, const Dims& dm, int cp, bool lce,
+                                                const float2* wv, float2 bias2) {
+    float2 acc[BR][WS];
+#pragma unroll
+    for (int r = 0; r < BR; ++r)
+#pragma unroll
+        for (int c = 0; c < WS; ++c) acc[r][c] = bias2;
+    const int y = y0 + r0, x = x0;
+    if (lce) {
+        const bool inside = y >= 2 && y + BR + 1 < dm.H && x >= 2 && x + WS + 1 < dm.W;
+        if (inside) lce_block<WS, BR, false>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wv, acc);
+        else        lce_block<WS, BR, true>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wv, acc);
+    }
+#pragma unroll
+    for (int r = 0; r < BR; ++r)
+#pragma unroll
+        for (int c = 0; c < WS; ++c) {
+            const float2 att = *reinterpret_cast<const float2*>(stage_o + ((r0 + r) * WS + c) * 32 + 2 * cp);
+            const float2 r2 = __fadd2_rn(att, acc[r][c]);
+            outb[((size_t)(y + r) * dm.W + x + c) * (dm.C / 2)] = pack2_bf16(r2.x, r2.y);
+        }
+}
+
+__global__ void __launch_bounds__(img::MAX_WARPS * 32, 2)
+attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
+                  const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
+                  const float* __restrict__ lce_w, const float* __restrict__ lce_b,
+                  __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
+                  int32_t* __restrict__ status, Dims dm, ImgGeom gm) {
+    using namespace img;
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t sbase = smem_u32(smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nthreads = gm.nw * 32;
+    const int h = blockIdx.x % dm.heads, b = blockIdx.x / dm.heads;
+    const size_t tok_bytes = (size_t)dm.C * 2;
+    const size_t row_bytes = (size_t)dm.W * tok_bytes;
+    const size_t img_off = (size_t)b * dm.H * row_bytes + (size_t)h * 64;    // this head's 32 channels
+    const uint8_t* Qb = reinterpret_cast<const uint8_t*>(Qg) + img_off;
+    const uint8_t* Kb = reinterpret_cast<const uint8_t*>(Kg) + img_off;
+    const uint8_t* Vb = reinterpret_cast<const uint8_t*>(Vg) + img_off;
+
+    // ---- 1. the head's K and V slices of the whole image (inputs of the call: no need to wait
+    //         for the routing kernel this launch may overlap) ----
+    for (int c = tid; c < dm.N * 4; c += nthreads) {
+        const int tok = c >> 2, q = c & 3;
+        const uint32_t dst = tok * 64 + ((q ^ ((tok >> 1) & 3)) << 4);
+        const size_t src = (size_t)tok * tok_bytes + q * 16;
+        cp_async_16(sbase + gm.off_k + dst, Kb + src, 16);
+        cp_async_16(sbase + gm.off_v + dst, Vb + src, 16);
+    }
+    cp_async_commit();
+    // LCE weights of the head as [tap][channel pair] (read back conflict-free)
+    if (dm.lce) {
+        const float* wp = lce_w + (size_t)h * 32 * 25;
+        for (int idx = tid; idx < 25 * 16; idx += nthreads) {
+            const int q = idx >> 4, cp = idx & 15;
+            *reinterpret_cast<float2*>(smem + gm.off_w + idx * 8) =
+                make_float2(__ldg(wp + (2 * cp) * 25 + q), __ldg(wp + (2 * cp + 1) * 25 + q));
+        }
+    }
+    pdl_wait();          // the index may come from the routing kernel this launch overlaps
+    // routing rows of this (image, head): coherent loads, checked once
+    int32_t* s_idx = reinterpret_cast<int32_t*>(smem + gm.off_idx);
+    {
+        const int hi = dm.heads_i == 1 ? 0 : h;
+        const int32_t* ib = index + ((size_t)b * dm.heads_i + hi) * dm.R * dm.topk;
+        for (int e = tid; e < dm.R * dm.topk; e += nthreads) {
+            int r = __ldcg(ib + e);
+            if (r < 0 || r >= dm.R) { record_error(status, BRA_ERR_INDEX, r); r = -1; }
+            s_idx[e] = r;
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+
+    // ---- 2. units of 16 query tokens, one warp each ----
+    const int g = lane >> 2, tq = lane & 3;                           // fragment row / column pair
+    const float sl2 = dm.scale * 1.4426950408889634f;
+    const int total_keys = dm.topk * dm.n_r;
+    const uint32_t kbase = sbase + gm.off_k, vbase = sbase + gm.off_v;
+    float* stage_o = reinterpret_cast<float*>(smem + gm.off_st) + warp * 16 * 32;   // [16 tokens][32 ch]
+    const int cp = lane & 15;                                         // LCE: channels 2cp, 2cp + 1 of this head
+    const int run = (dm.ws & 1) ? 1 : 2;                              // LCE: tokens per thread step, along x
+    float2 bias2 = make_float2(0.f, 0.f);
+    if (lce_b) bias2 = make_float2(__ldg(lce_b + h * 32 + 2 * cp), __ldg(lce_b + h * 32 + 2 * cp + 1));
+    uint32_t* outb = reinterpret_cast<uint32_t*>(O) + img_off / 4 + cp;
+
+    for (int u = warp; u < gm.units; u += gm.nw) {
+        const int i = fdiv(u, gm.tpr, gm.mul_tpr);
+        const int t0 = (u - i * gm.tpr) * 16;
+        const int rows = min(16, dm.n_r - t0);
+        const int ry = fdiv(i, dm.S, gm.mul_s), rx = i - ry * dm.S;
+        const int y0 = ry * dm.hs, x0 = rx * dm.ws;                   // region origin in the map
+        const int32_t* irow = s_idx + i * dm.topk;
+
+        // A fragments of Q (rows g and g + 8 of the tile; rows beyond the region are zero)
+        uint32_t qa[2][4];
+        {
+            const int ta = t0 + g, tb = t0 + g + 8;
+            const bool va = g < rows, vb = g + 8 < rows;
+            const int tya = fdiv(va ? ta : 0, dm.ws, gm.mul_ws), txa = (va ? ta : 0) - tya * dm.ws;
+            const int tyb = fdiv(vb ? tb : 0, dm.ws, gm.mul_ws), txb = (vb ? tb : 0) - tyb * dm.ws;
+            const uint8_t* pa = Qb + (size_t)(y0 + tya) * row_bytes + (size_t)(x0 + txa) * tok_bytes + 4 * tq;
+            const uint8_t* pb = Qb + (size_t)(y0 + tyb) * row_bytes + (size_t)(x0 + txb) * tok_bytes + 4 * tq;
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                qa[s][0] = va ? ldg_u32(pa + 32 * s) : 0u;
+                qa[s][1] = vb ? ldg_u32(pb + 32 * s) : 0u;
+                qa[s][2] = va ? ldg_u32(pa + 32 * s + 16) : 0u;
+                qa[s][3] = vb ? ldg_u32(pb + 32 * s + 16) : 0u;
+            }
+        }
+        const bool lower_only = rows <= 8;                            // rows g + 8 are padding
+
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        float o[4][4];
+#pragma unroll
+        for (int n = 0; n < 4; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) o[n][e] = 0.f;
+
+        for (int blk = 0; blk < gm.nblocks; ++blk) {
+            // token (= shared-memory row) of keys blk * 64 + lane and + 32; the other lanes fetch them by shuffle
+            int trow[2];
+            uint32_t vm[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int kk = blk * KB + lane + 32 * e;
+                bool valid = kk < total_keys;
+                int tr = 0;
+                if (valid) {
+                    const int m = fdiv(kk, dm.n_r, gm.mul_nr), t = kk - m * dm.n_r;
+                    const int r = irow[m];
+                    valid = r >= 0;
+                    if (valid) {
+                        const int qy = fdiv(r, dm.S, gm.mul_s), qx = r - qy * dm.S;
+                        const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
+                        tr = (qy * dm.hs + ty) * dm.W + qx * dm.ws + tx;
+                    }
+                }
+                trow[e] = tr;
+                vm[e] = __ballot_sync(0xffffffffu, valid);
+            }
+            if ((vm[0] | vm[1]) == 0u) continue;                      // nothing in this block counts
+            // S = Q K^T: 8 key tiles of 8
+            float c[8][4];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
+                uint32_t kb[4];
+                const int tr = __shfl_sync(0xffffffffu, trow[j >> 2], ((8 * j) & 31) + (lane & 7));
+                const int q = lane >> 3;                              // channel chunk of this lane's matrix
+                ldmatrix_x4(kbase + tr * 64 + ((q ^ ((tr >> 1) & 3)) << 4), kb);
+                mma_bf16(c[j], qa[0], kb[0], kb[1]);
+                mma_bf16(c[j], qa[1], kb[2], kb[3]);
+            }
+            // keys that do not count (padding of the last block, out-of-range entries): -inf
+            if ((vm[0] & vm[1]) != 0xffffffffu) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t bits = vm[j >> 2] >> (((8 * j) & 31) + 2 * tq);
+                    if (!(bits & 1u)) { c[j][0] = -INFINITY; c[j][2] = -INFINITY; }
+                    if (!(bits & 2u)) { c[j][1] = -INFINITY; c[j][3] = -INFINITY; }
+                }
+            }
+            // online softmax on rows g (elements 0, 1) and g + 8 (elements 2, 3)
+            float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                mx[0] = fmax3(mx[0], c[j][0], c[j][1]);
+                mx[1] = fmax3(mx[1], c[j][2], c[j][3]);
+            }
+            float corr[2], mneg[2];
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+                const float mnew = fmaxf(m_run[r], mx[r] * sl2);      // sl2 > 0
+                corr[r] = (mnew == -INFINITY) ? 1.f : ex2_approx(m_run[r] - mnew);
+                mneg[r] = (mnew == -INFINITY) ? 0.f : -mnew;
+                m_run[r] = mnew;
+                l_run[r] *= corr[r];
+            }
+#pragma unroll
+            for (int n = 0; n < 4; ++n) { o[n][0] *= corr[0]; o[n][1] *= corr[0]; o[n][2] *= corr[1]; o[n][3] *= corr[1]; }
+            uint32_t pa[4][4];                                        // P as A fragments: 4 k-steps of 16 keys
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float p0 = ex2_approx(fmaf(c[j][0], sl2, mneg[0]));
+                const float p1 = ex2_approx(fmaf(c[j][1], sl2, mneg[0]));
+                float p2 = 0.f, p3 = 0.f;
+                if (!lower_only) {
+                    p2 = ex2_approx(fmaf(c[j][2], sl2, mneg[1]));
+                    p3 = ex2_approx(fmaf(c[j][3], sl2, mneg[1]));
+                }
+                l_run[0] += p0 + p1;
+                l_run[1] += p2 + p3;
+                pa[j >> 1][(j & 1) * 2] = pack2_bf16(p0, p1);
+                pa[j >> 1][(j & 1) * 2 + 1] = pack2_bf16(p2, p3);
+            }
+            // O += P V: 4 k-steps of 16 keys x 4 channel tiles of 8
+#pragma unroll
+            for (int s = 0; s < 4; ++s) {
+                const int tr = __shfl_sync(0xffffffffu, trow[s >> 1], ((16 * s) & 31) + (lane & 7) + ((lane >> 3) & 1) * 8);
+#pragma unroll
+                for (int np = 0; np < 2; ++np) {
+                    uint32_t vb[4];
+                    const int q = 2 * np + (lane >> 4);
+                    ldmatrix_x4_trans(vbase + tr * 64 + ((q ^ ((tr >> 1) & 3)) << 4), vb);
+                    mma_bf16(o[2 * np], pa[s], vb[0], vb[1]);
+                    mma_bf16(o[2 * np + 1], pa[s], vb[2], vb[3]);
+                }
+            }
+        }
+
+        // ---- 3. normalise; park O^att (fp32, this warp's tile); lse ----
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const int row = g + 8 * r;
+            if (row < rows) {
+                const float inv = l_run[r] > 0.f ? 1.f / l_run[r] : 0.f;
+#pragma unroll
+                for (int n = 0; n < 4; ++n)
+                    *reinterpret_cast<float2*>(stage_o + row * 32 + 8 * n + 2 * tq) =
+                        make_float2(o[n][2 * r] * inv, o[n][2 * r + 1] * inv);
+                if (lse && tq == 0) {
+                    const int t = t0 + row;
+                    const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
+                    lse[((size_t)b * dm.heads + h) * dm.N + (size_t)(y0 + ty) * dm.W + x0 + tx] =
+                        (m_run[r] + log2f(l_run[r])) * 0.6931471805599453f;
+                }
+            }
+        }
+        __syncwarp();
+
+        // ---- LCE + store: lane = (channel pair, every other run of `run` tokens along x) ----
+        {
+            float2 wv[25];
+            if (dm.lce) {
+#pragma unroll
+                for (int q = 0; q < 25; ++q) wv[q] = lds_f32x2(sbase + gm.off_w + (q * 16 + cp) * 8);
+            }
+            const uint32_t vcol = (cp & 3) * 4;
+            const int cq = cp >> 2;
+            // the two region shapes of the late stages: whole rows per half-warp, one shared window
+            const bool blk44 = dm.ws == 4 && rows == 16, blk22 = dm.ws == 2 && rows == 4;
+            if (blk44) lce_store_block<4, 2>(vbase, stage_o, outb, 2 * (lane >> 4), y0, x0, dm, cp, dm.lce, wv, bias2);
+            if (blk22) lce_store_block<2, 1>(vbase, stage_o, outb, lane >> 4, y0, x0, dm, cp, dm.lce, wv, bias2);
+            const int nruns = (blk44 || blk22) ? 0 : rows / run;      // tiles start at multiples of 16, n_r is a multiple of run
+            for (int u2 = lane >> 4; u2 < nruns; u2 += 2) {
+                const int t = t0 + u2 * run;
+                const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
+                const int y = y0 + ty, x = x0 + tx;
+                float2 acc[2] = {bias2, bias2};
+                if (dm.lce) {
+                    const bool inside = y >= 2 && y + 2 < dm.H && x >= 2 && x + run + 1 < dm.W;
+#pragma unroll
+                    for (int ti = 0; ti < 5; ++ti) {
+                        const int yy = y + ti - 2;
+                        float2 v[6];
+#pragma unroll
+                        for (int xx = 0; xx < 6; ++xx) {
+                            if (xx < run + 4) {
+                                const int xc = x + xx - 2;
+                                uint32_t w = 0u;
+                                if (inside || ((unsigned)yy < (unsigned)dm.H && (unsigned)xc < (unsigned)dm.W)) {
+                                    const int tok = yy * dm.W + xc;
+                                    w = lds_u32(vbase + tok * 64 + ((cq ^ ((tok >> 1) & 3)) << 4) + vcol);
+                                }
+                                v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+                            }
+                        }
+#pragma unroll
+                        for (int tj = 0; tj < 5; ++tj) {
+                            acc[0] = __ffma2_rn(wv[ti * 5 + tj], v[tj], acc[0]);
+                            if (run == 2) acc[1] = __ffma2_rn(wv[ti * 5 + tj], v[tj + 1], acc[1]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    if (e < run) {
+                        const float2 att = *reinterpret_cast<const float2*>(stage_o + (t - t0 + e) * 32 + 2 * cp);
+                        const float2 r2 = __fadd2_rn(att, acc[e]);
+                        outb[((size_t)y * dm.W + x + e) * (dm.C / 2)] = pack2_bf16(r2.x, r2.y);
+                    }
+                }
+            }
+        }
+        __syncwarp();                                                 // the staging tile is read: next unit may overwrite it
+    }
+}
+
+// ------------------------------------------------------------------ host side
+static ImgGeom img_geom(const Dims& d, int nw) {
+    ImgGeom g;
+    g.nw = nw;
+    g.tpr = (d.n_r + 15) / 16;
+    g.units = d.R * g.tpr;
+    g.nblocks = (d.topk * d.n_r + img::KB - 1) / img::KB;
+    g.mul_nr = recip32(d.n_r); g.mul_ws = recip32(d.ws); g.mul_s = recip32(d.S); g.mul_tpr = recip32(g.tpr);
+    int off = 0;
+    g.off_k = off;   off += d.N * 64;
+    g.off_v = off;   off += d.N * 64;
+    g.off_st = off;  off += nw * 2048;
+    g.off_w = off;   off += 25 * 16 * 8;
+    g.off_idx = off; off += ((d.R * d.topk * 4 + 15) / 16) * 16;
+    g.smem_bytes = off;
+    return g;
+}
+
+static int img_sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 1;
+    return n;
+}
+
+bool attend_img_supported(const Dims& d, int dtype) {
+    if (dtype != BRA_BF16 || d.d != 32) return false;
+    if ((long long)d.R * d.topk > img::MAX_ENTRIES || d.N > 4096) return false;
+    if ((d.ws & 1) == 0 && (d.n_r & 1)) return false;
+    if ((long long)d.topk * d.n_r * d.n_r >= (1ll << 32) || d.R > 65535 || d.n_r > 65535) return false;
+    if ((long long)d.B * d.heads >= (1ll << 31)) return false;
+    return img_geom(d, 1).smem_bytes <= 200 * 1024;
+}
+
+cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
+                              const int32_t* index, const float* lce_w, const float* lce_b,
+                              void* O, float* lse, int32_t* status, cudaStream_t st) {
+    // warps per CTA: the most that still lets every CTA of the grid be resident at once; if no
+    // choice does, the one with the most warps per SM
+    const long long grid = (long long)d.B * d.heads;
+    const int sms = img_sm_count();
+    static int smem_set = 0;
+    int best_nw = 0, best_warps = -1;
+    for (int nw = img::MAX_WARPS; nw >= 1; --nw) {
+        const ImgGeom g = img_geom(d, nw);
+        if (g.smem_bytes > 200 * 1024) continue;
+        if (g.smem_bytes > smem_set) {
+            cudaError_t e = cudaFuncSetAttribute(attend_img_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
+            if (e != cudaSuccess) return e;
+            smem_set = g.smem_bytes;
+        }
+        int occ = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, attend_img_kernel, nw * 32, g.smem_bytes) != cudaSuccess)
+            return cudaErrorUnknown;
+        if (occ <= 0) continue;
+        if ((long long)occ * sms >= grid) { best_nw = nw; break; }
+        if (occ * nw > best_warps) { best_warps = occ * nw; best_nw = nw; }
+    }
+    if (!best_nw) return cudaErrorInvalidConfiguration;
+    const ImgGeom g = img_geom(d, best_nw);
+    cudaError_t e = launch_kernel(attend_img_kernel, dim3((unsigned)grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st,
+                                  take_after_own_kernel(),
+                                  static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
+                                  static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b,
+                                  static_cast<__nv_bfloat16*>(O), lse, status, d, g);
+    count_launch();
+    return e;
+}
+
+}  // namespace bra

@@ -39,7 +39,7 @@ static bra_status make_dims(const bra_problem* p, Dims* out) {
     if (p->topk < 1 || (int64_t)p->topk > (int64_t)p->S * p->S) return BRA_ERR_TOPK;
     if (p->dtype != BRA_F32 && p->dtype != BRA_BF16) return BRA_ERR_DTYPE;
     if (p->lce_ksize != 0 && p->lce_ksize != 5) return BRA_ERR_UNSUPPORTED;
-    if (p->impl < BRA_IMPL_AUTO || p->impl > BRA_IMPL_TC) return BRA_ERR_UNSUPPORTED;
+    if (p->impl < BRA_IMPL_AUTO || p->impl > BRA_IMPL_IMG) return BRA_ERR_UNSUPPORTED;
     Dims d;
     d.B = p->B; d.H = p->H; d.W = p->W; d.C = p->C; d.heads = p->heads; d.S = p->S; d.topk = p->topk;
     d.d = p->C / p->heads;
@@ -74,7 +74,7 @@ static bra_status check_ws(const Dims& d, const void* ws, size_t ws_bytes, WsLay
     return BRA_OK;
 }
 
-enum Path { PATH_NONE, PATH_SIMT, PATH_MMA, PATH_TC, PATH_TC_WIDE };
+enum Path { PATH_NONE, PATH_SIMT, PATH_MMA, PATH_TC, PATH_TC_WIDE, PATH_IMG };
 
 static Path choose_attend(const Dims& d, int dtype, int impl) {
     switch (impl) {
@@ -82,10 +82,13 @@ static Path choose_attend(const Dims& d, int dtype, int impl) {
         case BRA_IMPL_MMA:  return attend_mma_supported(d, dtype) ? PATH_MMA : PATH_NONE;
         case BRA_IMPL_TC:   return attend_tc_supported(d, dtype) ? PATH_TC
                                  : attend_tc_wide_supported(d, dtype) ? PATH_TC_WIDE : PATH_NONE;
+        case BRA_IMPL_IMG:  return attend_img_supported(d, dtype) ? PATH_IMG : PATH_NONE;
         default: break;
     }
     if (attend_tc_supported(d, dtype)) return PATH_TC;
     if (attend_tc_wide_supported(d, dtype)) return PATH_TC_WIDE;
+    // one CTA per (image, head): worth it once those fill a good part of the GPU
+    if (attend_img_supported(d, dtype) && (long long)d.B * d.heads >= 64) return PATH_IMG;
     if (attend_mma_supported(d, dtype)) return PATH_MMA;
     if (attend_simt_supported(d)) return PATH_SIMT;
     return PATH_NONE;
@@ -108,6 +111,7 @@ static bra_status run_attend(Path path, const Dims& d, int dtype, const void* Q,
         case PATH_MMA:  e = launch_attend_mma(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
         case PATH_TC:   e = launch_attend_tc(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
         case PATH_TC_WIDE: e = launch_attend_tc_wide(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
+        case PATH_IMG:  e = launch_attend_img(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
         default: return BRA_ERR_UNSUPPORTED;
     }
     return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;

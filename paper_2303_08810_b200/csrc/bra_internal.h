@@ -75,6 +75,10 @@ cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const 
                              const int32_t* index, const float* lce_w, const float* lce_b,
                              void* O, float* lse, int32_t* status, cudaStream_t st);
 
+bool attend_img_supported(const Dims& d, int dtype);
+cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
+                              const int32_t* index, const float* lce_w, const float* lce_b,
+                              void* O, float* lse, int32_t* status, cudaStream_t st);
 bool attend_tc_wide_supported(const Dims& d, int dtype);
 cudaError_t launch_attend_tc_wide(const Dims& d, const void* Q, const void* K, const void* V,
                                   const int32_t* index, const float* lce_w, const float* lce_b,

@@ -147,7 +147,7 @@ def test_route_exact_ties_go_to_lower_region(bra):
 
 
 # ------------------------------------------------------------------ attention
-IMPLS = {"simt": 1, "mma": 2, "tc": 3, "auto": 0}
+IMPLS = {"simt": 1, "mma": 2, "tc": 3, "img": 4, "auto": 0}
 
 
 def run_attend_case(bra, cfg, impl, seed, shared=False, lce=True, bias=False, scale=0.0,
@@ -182,7 +182,7 @@ def run_attend_case(bra, cfg, impl, seed, shared=False, lce=True, bias=False, sc
     return O
 
 
-@pytest.mark.parametrize("impl", ["simt", "mma", "tc", "auto"])
+@pytest.mark.parametrize("impl", ["simt", "mma", "tc", "img", "auto"])
 @pytest.mark.parametrize("n", [1, 2, 3, 4, 5])
 def test_attend_matches_oracle_on_benchmark_configs(bra, n, impl):
     run_attend_case(bra, CONFIGS[n], impl, seed=1000 + n)
@@ -254,6 +254,33 @@ def test_attend_mma_options(bra):
     run_attend_case(bra, cfg, "mma", seed=6, index=idx)
 
 
+# head dim 32, bf16, maps small enough that one (image, head) of K and V fits in shared memory
+IMG_CASES = [c for c in MMA_CASES if c.H * c.W <= 1500] + [
+    BraConfig("img-tail-tile-n_r=24", 2, 12, 16, 64, 2, 2, 3, "bf16"),
+    BraConfig("img-5x5-regions-odd", 1, 15, 15, 32, 1, 3, 4, "bf16"),
+    BraConfig("img-k-many-blocks", 1, 16, 16, 64, 2, 4, 16, "bf16"),
+    BraConfig("img-many-images", 40, 14, 14, 64, 2, 7, 5, "bf16"),
+]
+
+
+@pytest.mark.parametrize("cfg", IMG_CASES, ids=[c.name for c in IMG_CASES])
+def test_attend_img_shapes(bra, cfg):
+    run_attend_case(bra, cfg, "img", seed=24)
+
+
+def test_attend_img_options(bra):
+    cfg = BraConfig("img-opts", 2, 16, 16, 64, 2, 4, 3, "bf16")
+    run_attend_case(bra, cfg, "img", seed=6, lce=False)
+    run_attend_case(bra, cfg, "img", seed=6, bias=True)
+    run_attend_case(bra, cfg, "img", seed=6, scale=0.5)
+    run_attend_case(bra, cfg, "img", seed=6, shared=True)
+    run_attend_case(bra, cfg, "img", seed=6, clustered=True)
+    rng = np.random.default_rng(3)
+    idx = rng.integers(0, cfg.R, size=(cfg.B, cfg.heads, cfg.R, cfg.topk)).astype(np.int32)
+    idx[0, 0, 0] = [5, 5, 5]
+    run_attend_case(bra, cfg, "img", seed=6, index=idx)
+
+
 # head dim 32, regions 16 tokens wide and a multiple of 8 high: the tcgen05 kernel for large regions
 TC_WIDE_CASES = [
     BraConfig("wide-16x16-k4", 2, 32, 32, 64, 2, 2, 4, "bf16"),
@@ -299,7 +326,7 @@ def test_attend_options(bra, impl, cfg):
 
 
 @pytest.mark.parametrize("hw", [16, 32])
-@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("impl", ["simt", "img", "auto"])
 def test_out_of_range_index_is_reported_not_fatal(bra, impl, hw):
     import torch
     cfg = BraConfig("bad-index", 1, hw, hw, 64, 2, 4, 2, "bf16")
