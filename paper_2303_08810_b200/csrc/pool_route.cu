@@ -103,7 +103,7 @@ __device__ __forceinline__ uint32_t ordered_bits(float s) {
 }
 
 constexpr int ROWS_PER_CTA = 8;
-constexpr int SELECT_MAX_K = 8;             // up to here k rounds of a warp maximum beat the full sort
+constexpr int SELECT_MAX_K = 32;            // up to here k rounds of a warp maximum beat the full sort
 
 template <int E>   // E score slots per lane: handles R <= 32 * E
 __global__ void __launch_bounds__(256)
@@ -159,36 +159,23 @@ route_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ ind
             key[e] = j < dm.R ? ((unsigned long long)ordered_bits(acc[e]) << 32) | (0xffffffffu - (uint32_t)j)
                               : 0ull;
         }
-        if (dm.topk == 1) {
-            // the row maximum is all that is asked for: one warp reduction
-            unsigned long long best = key[0];
-#pragma unroll
-            for (int e = 1; e < E; ++e) best = key[e] > best ? key[e] : best;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-                best = other > best ? other : best;
-            }
-            if (lane == 0)
-                index[((size_t)b * dm.heads_i + h) * dm.R + i] = (int32_t)(0xffffffffu - (uint32_t)(best & 0xffffffffull));
-            continue;
-        }
         int32_t* out = index + (((size_t)b * dm.heads_i + h) * dm.R + i) * dm.topk;
         if (dm.topk <= SELECT_MAX_K) {
-            // a few winners: one warp-wide maximum per rank, the winner's key cleared for the next round
+            // a few winners: one warp-wide maximum per rank (score bits first, then, among the lanes that
+            // hold that score, the lower region), the winner's key cleared for the next round
             for (int m = 0; m < dm.topk; ++m) {
                 unsigned long long best = key[0];
 #pragma unroll
                 for (int e = 1; e < E; ++e) best = key[e] > best ? key[e] : best;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-                    best = other > best ? other : best;
-                }
+                const uint32_t hi = (uint32_t)(best >> 32);
+                const uint32_t top_hi = __reduce_max_sync(0xffffffffu, hi);
+                const uint32_t lo = hi == top_hi ? (uint32_t)best : 0u;
+                const uint32_t top_lo = __reduce_max_sync(0xffffffffu, lo);
+                const unsigned long long top = ((unsigned long long)top_hi << 32) | top_lo;
 #pragma unroll
                 for (int e = 0; e < E; ++e)
-                    if (key[e] == best) key[e] = 0ull;       // keys are distinct: they carry the region number
-                if (lane == 0) out[m] = (int32_t)(0xffffffffu - (uint32_t)(best & 0xffffffffull));
+                    if (key[e] == top) key[e] = 0ull;        // keys are distinct: they carry the region number
+                if (lane == 0) out[m] = (int32_t)(0xffffffffu - top_lo);
             }
             continue;
         }
