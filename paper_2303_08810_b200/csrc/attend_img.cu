@@ -106,7 +106,9 @@ __device__ __forceinline__ void lce_store_block(uint32_t vbase, const float* sta
         }
 }
 
-__global__ void __launch_bounds__(img::MAX_WARPS * 32, 2)
+// SMALL: CTAs of up to 5 warps (two per SM by shared memory): room for ~200 registers per thread.
+template <bool SMALL>
+__global__ void __launch_bounds__(SMALL ? 160 : img::MAX_WARPS * 32, 2)
 attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
                   const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
                   const float* __restrict__ lce_w, const float* __restrict__ lce_b,
@@ -145,7 +147,7 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
         }
     }
     pdl_wait();          // the index may come from the routing kernel this launch overlaps
-    // routing rows of this (image, head): coherent loads, checked once
+    // routing rows of this (image, head): coherent loads, checked once, kept as token ids (-1: bad entry)
     int32_t* s_idx = reinterpret_cast<int32_t*>(smem + gm.off_idx);
     {
         const int hi = dm.heads_i == 1 ? 0 : h;
@@ -153,6 +155,10 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
         for (int e = tid; e < dm.R * dm.topk; e += nthreads) {
             int r = __ldcg(ib + e);
             if (r < 0 || r >= dm.R) { record_error(status, BRA_ERR_INDEX, r); r = -1; }
+            if (r >= 0) {                        // keep the token id of the routed region's first token
+                const int qy = fdiv(r, dm.S, gm.mul_s), qx = r - qy * dm.S;
+                r = qy * dm.hs * dm.W + qx * dm.ws;
+            }
             s_idx[e] = r;
         }
     }
@@ -170,6 +176,20 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
     float2 bias2 = make_float2(0.f, 0.f);
     if (lce_b) bias2 = make_float2(__ldg(lce_b + h * 32 + 2 * cp), __ldg(lce_b + h * 32 + 2 * cp + 1));
     uint32_t* outb = reinterpret_cast<uint32_t*>(O) + img_off / 4 + cp;
+
+    // key kk = blk * 64 + lane + 32 e of a unit is token t = kk mod n_r of routed entry m = kk / n_r.
+    // When n_r divides 64 a lane sees the same t in every block: its offset inside the region is fixed.
+    const bool fixed_t = (KB % dm.n_r) == 0;
+    const int mstep = KB / dm.n_r;
+    int m_of[2], toff[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int kk = lane + 32 * e;
+        m_of[e] = fdiv(kk, dm.n_r, gm.mul_nr);
+        const int t = kk - m_of[e] * dm.n_r;
+        const int ty = fdiv(t, dm.ws, gm.mul_ws);
+        toff[e] = ty * dm.W + (t - ty * dm.ws);
+    }
 
     for (int u = warp; u < gm.units; u += gm.nw) {
         const int i = fdiv(u, gm.tpr, gm.mul_tpr);
@@ -215,14 +235,19 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
                 bool valid = kk < total_keys;
                 int tr = 0;
                 if (valid) {
-                    const int m = fdiv(kk, dm.n_r, gm.mul_nr), t = kk - m * dm.n_r;
-                    const int r = irow[m];
-                    valid = r >= 0;
-                    if (valid) {
-                        const int qy = fdiv(r, dm.S, gm.mul_s), qx = r - qy * dm.S;
-                        const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
-                        tr = (qy * dm.hs + ty) * dm.W + qx * dm.ws + tx;
+                    int m, off;
+                    if (fixed_t) {
+                        m = blk * mstep + m_of[e];
+                        off = toff[e];
+                    } else {
+                        m = fdiv(kk, dm.n_r, gm.mul_nr);
+                        const int t = kk - m * dm.n_r;
+                        const int ty = fdiv(t, dm.ws, gm.mul_ws);
+                        off = ty * dm.W + (t - ty * dm.ws);
                     }
+                    const int base = irow[m];
+                    valid = base >= 0;
+                    tr = valid ? base + off : 0;
                 }
                 trow[e] = tr;
                 vm[e] = __ballot_sync(0xffffffffu, valid);
@@ -267,23 +292,33 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
                 m_run[r] = mnew;
                 l_run[r] *= corr[r];
             }
+            const float2 corr0 = make_float2(corr[0], corr[0]), corr1 = make_float2(corr[1], corr[1]);
 #pragma unroll
-            for (int n = 0; n < 4; ++n) { o[n][0] *= corr[0]; o[n][1] *= corr[0]; o[n][2] *= corr[1]; o[n][3] *= corr[1]; }
+            for (int n = 0; n < 4; ++n) {
+                const float2 a = __fmul2_rn(make_float2(o[n][0], o[n][1]), corr0);
+                const float2 bq = __fmul2_rn(make_float2(o[n][2], o[n][3]), corr1);
+                o[n][0] = a.x; o[n][1] = a.y; o[n][2] = bq.x; o[n][3] = bq.y;
+            }
             uint32_t pa[4][4];                                        // P as A fragments: 4 k-steps of 16 keys
+            const float2 sl2v = make_float2(sl2, sl2);
+            const float2 mneg0 = make_float2(mneg[0], mneg[0]), mneg1 = make_float2(mneg[1], mneg[1]);
+            float2 sum0 = make_float2(0.f, 0.f), sum1 = make_float2(0.f, 0.f);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const float p0 = ex2_approx(fmaf(c[j][0], sl2, mneg[0]));
-                const float p1 = ex2_approx(fmaf(c[j][1], sl2, mneg[0]));
-                float p2 = 0.f, p3 = 0.f;
+                const float2 a0 = __ffma2_rn(make_float2(c[j][0], c[j][1]), sl2v, mneg0);
+                const float2 p01 = make_float2(ex2_approx(a0.x), ex2_approx(a0.y));
+                float2 p23 = make_float2(0.f, 0.f);
                 if (!lower_only) {
-                    p2 = ex2_approx(fmaf(c[j][2], sl2, mneg[1]));
-                    p3 = ex2_approx(fmaf(c[j][3], sl2, mneg[1]));
+                    const float2 a1 = __ffma2_rn(make_float2(c[j][2], c[j][3]), sl2v, mneg1);
+                    p23 = make_float2(ex2_approx(a1.x), ex2_approx(a1.y));
                 }
-                l_run[0] += p0 + p1;
-                l_run[1] += p2 + p3;
-                pa[j >> 1][(j & 1) * 2] = pack2_bf16(p0, p1);
-                pa[j >> 1][(j & 1) * 2 + 1] = pack2_bf16(p2, p3);
+                sum0 = __fadd2_rn(sum0, p01);
+                sum1 = __fadd2_rn(sum1, p23);
+                pa[j >> 1][(j & 1) * 2] = pack2_bf16(p01.x, p01.y);
+                pa[j >> 1][(j & 1) * 2 + 1] = pack2_bf16(p23.x, p23.y);
             }
+            l_run[0] += sum0.x + sum0.y;
+            l_run[1] += sum1.x + sum1.y;
             // O += P V: 4 k-steps of 16 keys x 4 channel tiles of 8
 #pragma unroll
             for (int s = 0; s < 4; ++s) {
@@ -416,37 +451,56 @@ bool attend_img_supported(const Dims& d, int dtype) {
     return img_geom(d, 1).smem_bytes <= 200 * 1024;
 }
 
+template <bool SMALL>
+static cudaError_t img_occupancy(int nw, int smem_bytes, int* occ) {
+    static int smem_set = 0;
+    if (smem_bytes > smem_set) {
+        cudaError_t e = cudaFuncSetAttribute(attend_img_kernel<SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        if (e != cudaSuccess) return e;
+        smem_set = smem_bytes;
+    }
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, attend_img_kernel<SMALL>, nw * 32, smem_bytes);
+}
+
 cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
                               const int32_t* index, const float* lce_w, const float* lce_b,
                               void* O, float* lse, int32_t* status, cudaStream_t st) {
     // warps per CTA: the most that still lets every CTA of the grid be resident at once; if no
-    // choice does, the one with the most warps per SM
+    // choice does, the one with the most warps per SM.  Remembered per shape.
     const long long grid = (long long)d.B * d.heads;
-    const int sms = img_sm_count();
-    static int smem_set = 0;
-    int best_nw = 0, best_warps = -1;
-    for (int nw = img::MAX_WARPS; nw >= 1; --nw) {
-        const ImgGeom g = img_geom(d, nw);
-        if (g.smem_bytes > 200 * 1024) continue;
-        if (g.smem_bytes > smem_set) {
-            cudaError_t e = cudaFuncSetAttribute(attend_img_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
+    static thread_local struct { long long grid; int N, ents, nw; } memo = {0, 0, 0, 0};
+    int best_nw = 0;
+    if (memo.nw && memo.grid == grid && memo.N == d.N && memo.ents == d.R * d.topk) {
+        best_nw = memo.nw;
+    } else {
+        const int sms = img_sm_count();
+        int best_warps = -1;
+        for (int nw = img::MAX_WARPS; nw >= 1; --nw) {
+            const ImgGeom g = img_geom(d, nw);
+            if (g.smem_bytes > 200 * 1024) continue;
+            int occ = 0;
+            const cudaError_t e = nw <= 5 ? img_occupancy<true>(nw, g.smem_bytes, &occ)
+                                          : img_occupancy<false>(nw, g.smem_bytes, &occ);
             if (e != cudaSuccess) return e;
-            smem_set = g.smem_bytes;
+            if (occ <= 0) continue;
+            if ((long long)occ * sms >= grid) { best_nw = nw; break; }
+            if (occ * nw > best_warps) { best_warps = occ * nw; best_nw = nw; }
         }
-        int occ = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, attend_img_kernel, nw * 32, g.smem_bytes) != cudaSuccess)
-            return cudaErrorUnknown;
-        if (occ <= 0) continue;
-        if ((long long)occ * sms >= grid) { best_nw = nw; break; }
-        if (occ * nw > best_warps) { best_warps = occ * nw; best_nw = nw; }
+        if (!best_nw) return cudaErrorInvalidConfiguration;
+        memo.grid = grid; memo.N = d.N; memo.ents = d.R * d.topk; memo.nw = best_nw;
     }
-    if (!best_nw) return cudaErrorInvalidConfiguration;
     const ImgGeom g = img_geom(d, best_nw);
-    cudaError_t e = launch_kernel(attend_img_kernel, dim3((unsigned)grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st,
-                                  take_after_own_kernel(),
-                                  static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
-                                  static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b,
-                                  static_cast<__nv_bfloat16*>(O), lse, status, d, g);
+    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(Q);
+    const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(K);
+    const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(V);
+    const bool pdl = take_after_own_kernel();
+    cudaError_t e;
+    if (best_nw <= 5)
+        e = launch_kernel(attend_img_kernel<true>, dim3((unsigned)grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st, pdl,
+                          q, k, v, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, g);
+    else
+        e = launch_kernel(attend_img_kernel<false>, dim3((unsigned)grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st, pdl,
+                          q, k, v, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, g);
     count_launch();
     return e;
 }
