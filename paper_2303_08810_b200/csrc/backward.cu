@@ -12,6 +12,7 @@
 //   4. d_lce_w / d_lce_b: per-CTA partial sums, then a fixed-order final sum.
 // Steps 2 and 3 run on the tensor cores instead (backward_mma.cu) for bf16 with head dim 32.
 #include "bra_internal.h"
+#include "sm100_ptx.cuh"
 
 namespace bra {
 
@@ -225,83 +226,175 @@ template <> struct RawPair<__nv_bfloat16> {
         return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
     }
 };
-constexpr int DW_SLOTS = 4;     // row slots (blockDim.y)
+constexpr int DW_TI = 5;        // tap rows (blockDim.y)
 constexpr int DW_CP = 64;       // channel pairs per pass (blockDim.x at most)
 
+// Partial LCE weight gradient of a strip of rows_per_block image rows:
+//   dw[c, ti, tj] += dO[b, y, x, c] * V[b, y + ti - 2, x + tj - 2, c]   (and db[c] += dO)
+// Thread = (channel pair, tap row ti): it walks the strip's output rows and, along x, keeps the
+// five V values of its tap row under the sliding window in registers (one new load per step),
+// so its five sums (tj) take one dO load, one V load and five FMAs per position.  No sums are
+// shared between threads: nothing to reduce inside the CTA, and the order of additions is fixed
+// (rows ascending, x ascending).  Few registers, many warps: the loads of other warps hide the
+// latency of this one's.
 template <typename T>
-__global__ void __launch_bounds__(DW_CP * DW_SLOTS)
+__global__ void __launch_bounds__(DW_CP * DW_TI)
 bwd_dw_partial_kernel(const T* __restrict__ V, const T* __restrict__ dO, float* __restrict__ part,
                       int rows_per_block, Dims dm) {
-    extern __shared__ float2 red[];   // [blockDim.x][26]
+    typedef typename RawPair<T>::type raw_t;
     const long long rows = (long long)dm.B * dm.H;
     const long long r0 = (long long)blockIdx.x * rows_per_block;
     const long long r1 = r0 + rows_per_block < rows ? r0 + rows_per_block : rows;
     const int pairs = dm.C >> 1;
+    const int ti = threadIdx.y;
+    const size_t tokp = (size_t)dm.C;                      // elements per token
     for (int cp0 = 0; cp0 < pairs; cp0 += blockDim.x) {
         const int cp = cp0 + threadIdx.x;
-        const bool active = cp < pairs;
-        float2 acc[26];
+        if (cp >= pairs) continue;
+        float2 acc[5], accb = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < 26; ++k) acc[k] = make_float2(0.f, 0.f);
-        if (active) {
-            const long long rowp = (long long)dm.W * dm.C;
-            for (long long r = r0 + threadIdx.y; r < r1; r += DW_SLOTS) {
-                const int b = (int)(r / dm.H), y = (int)(r - (long long)b * dm.H);
-                const T* vimg = V + (size_t)b * dm.N * dm.C + 2 * cp;
-                const T* grow = dO + ((size_t)b * dm.N + (size_t)y * dm.W) * dm.C + 2 * cp;
-                const T* vrow[5];
-                bool rv[5];
+        for (int k = 0; k < 5; ++k) acc[k] = make_float2(0.f, 0.f);
+        for (long long r = r0; r < r1; ++r) {
+            const int b = (int)(r / dm.H), y = (int)(r - (long long)b * dm.H);
+            const int yy = y + ti - 2;
+            if (yy < 0 || yy >= dm.H) continue;            // this tap row reads zeros for this output row
+            const T* grow = dO + ((size_t)b * dm.N + (size_t)y * dm.W) * tokp + 2 * cp;
+            const T* vrow = V + ((size_t)b * dm.N + (size_t)yy * dm.W) * tokp + 2 * cp;
+            // window w[k] = V[yy][x + k - 2]; before x = 0: columns -2, -1 are zero, 0 and 1 are loaded
+            float2 w0 = make_float2(0.f, 0.f), w1 = w0;
+            float2 w2 = RawPair<T>::unpack(RawPair<T>::load(vrow));
+            float2 w3 = RawPair<T>::unpack(dm.W > 1 ? RawPair<T>::load(vrow + tokp) : RawPair<T>::zero());
+            for (int x0 = 0; x0 < dm.W; x0 += 4) {
+                // four positions per trip: their loads go out together
+                raw_t nv[4], gr[4];
 #pragma unroll
-                for (int ti = 0; ti < 5; ++ti) {
-                    const int yy = y + ti - 2;
-                    rv[ti] = yy >= 0 && yy < dm.H;
-                    vrow[ti] = vimg + (long long)(rv[ti] ? yy : y) * rowp - 2 * dm.C;
+                for (int u = 0; u < 4; ++u) {
+                    const int x = x0 + u;
+                    nv[u] = x + 2 < dm.W ? RawPair<T>::load(vrow + (size_t)(x + 2) * tokp) : RawPair<T>::zero();
+                    gr[u] = x < dm.W ? RawPair<T>::load(grow + (size_t)x * tokp) : RawPair<T>::zero();
                 }
-                // G positions along x at a time: their 5 x (G + 4) window of V is loaded once (zeros
-                // outside the map), all loads in flight before the first FMA
-                constexpr int G = sizeof(T) == 2 ? 5 : 2;
-                typedef typename RawPair<T>::type raw_t;
-                for (int xb = 0; xb < dm.W; xb += G) {
-                    raw_t win[5][G + 4];
-                    raw_t gr[G];
 #pragma unroll
-                    for (int cc = 0; cc < G + 4; ++cc) {
-                        const bool cv = (unsigned)(xb + cc - 2) < (unsigned)dm.W;
-#pragma unroll
-                        for (int ti = 0; ti < 5; ++ti)
-                            win[ti][cc] = (rv[ti] && cv) ? RawPair<T>::load(vrow[ti] + (size_t)(xb + cc) * dm.C) : RawPair<T>::zero();
-                    }
-#pragma unroll
-                    for (int px = 0; px < G; ++px)
-                        gr[px] = xb + px < dm.W ? RawPair<T>::load(grow + (size_t)(xb + px) * dm.C) : RawPair<T>::zero();
-#pragma unroll
-                    for (int px = 0; px < G; ++px) {
-                        const float2 g = RawPair<T>::unpack(gr[px]);   // zero beyond the row: adds nothing
-                        acc[25] = __fadd2_rn(acc[25], g);
-#pragma unroll
-                        for (int ti = 0; ti < 5; ++ti)
-#pragma unroll
-                            for (int tj = 0; tj < 5; ++tj)
-                                acc[ti * 5 + tj] = __ffma2_rn(g, RawPair<T>::unpack(win[ti][px + tj]), acc[ti * 5 + tj]);
-                    }
+                for (int u = 0; u < 4; ++u) {
+                    const float2 w4 = RawPair<T>::unpack(nv[u]);
+                    const float2 g = RawPair<T>::unpack(gr[u]);    // zero beyond the row: adds nothing
+                    if (ti == 2) accb = __fadd2_rn(accb, g);
+                    acc[0] = __ffma2_rn(g, w0, acc[0]);
+                    acc[1] = __ffma2_rn(g, w1, acc[1]);
+                    acc[2] = __ffma2_rn(g, w2, acc[2]);
+                    acc[3] = __ffma2_rn(g, w3, acc[3]);
+                    acc[4] = __ffma2_rn(g, w4, acc[4]);
+                    w0 = w1; w1 = w2; w2 = w3; w3 = w4;
                 }
             }
         }
-        // row slots added in the order 0, 1, 2, ...
-        for (int slot = 0; slot < DW_SLOTS; ++slot) {
-            if ((int)threadIdx.y == slot && active) {
+        float* out = part + ((size_t)blockIdx.x * dm.C + 2 * cp) * 26;
 #pragma unroll
-                for (int k = 0; k < 26; ++k)
-                    red[threadIdx.x * 26 + k] = slot == 0 ? acc[k] : __fadd2_rn(red[threadIdx.x * 26 + k], acc[k]);
+        for (int k = 0; k < 5; ++k) { out[ti * 5 + k] = acc[k].x; out[26 + ti * 5 + k] = acc[k].y; }
+        if (ti == 2) { out[25] = accb.x; out[26 + 25] = accb.y; }
+    }
+}
+
+// a channel pair read from shared memory by 32-bit address, as two floats
+template <typename T> struct SmemPair;
+template <> struct SmemPair<float> {
+    static __device__ __forceinline__ float2 load(uint32_t a) { return ptx::lds_f32x2(a); }
+};
+template <> struct SmemPair<__nv_bfloat16> {
+    static __device__ __forceinline__ float2 load(uint32_t a) {
+        const uint32_t w = ptx::lds_u32(a);
+        return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    }
+};
+
+// The same sums with the strip's rows of V (rows_per_block + 4) and dO (rows_per_block) copied to
+// shared memory first: every byte of the strip is in flight at once, instead of one dependent round
+// of global loads per four positions.  Used when the rows fit.
+template <typename T>
+__global__ void __launch_bounds__(DW_CP * DW_TI)
+bwd_dw_partial_staged_kernel(const T* __restrict__ V, const T* __restrict__ dO, float* __restrict__ part,
+                             int rows_per_block, Dims dm) {
+    typedef typename RawPair<T>::type raw_t;
+    extern __shared__ __align__(16) uint8_t dw_smem[];
+    const long long rows = (long long)dm.B * dm.H;
+    const long long r0 = (long long)blockIdx.x * rows_per_block;
+    const long long r1 = r0 + rows_per_block < rows ? r0 + rows_per_block : rows;
+    const size_t row_elems = (size_t)dm.W * dm.C;
+    const int row_chunks = (int)(row_elems * sizeof(T) / 16);
+    T* Vs = reinterpret_cast<T*>(dw_smem);                              // slot s = image row r0 - 2 + s (row space of all images)
+    T* Gs = Vs + (size_t)(rows_per_block + 4) * row_elems;
+    const int tid = threadIdx.y * blockDim.x + threadIdx.x, nthreads = blockDim.x * blockDim.y;
+    const uint32_t vs_addr = ptx::smem_u32(Vs), gs_addr = ptx::smem_u32(Gs);
+    for (int s = 0; s < rows_per_block + 4; ++s) {
+        const long long rr = r0 - 2 + s;
+        if (rr < 0 || rr >= rows) continue;                             // never read: its tap rows are outside the map
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(V + (size_t)rr * row_elems);
+        for (int c = tid; c < row_chunks; c += nthreads)
+            ptx::cp_async_16(vs_addr + (uint32_t)(s * row_chunks + c) * 16, src + (size_t)c * 16, 16);
+    }
+    for (int s = 0; s < (int)(r1 - r0); ++s) {
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(dO + (size_t)(r0 + s) * row_elems);
+        for (int c = tid; c < row_chunks; c += nthreads)
+            ptx::cp_async_16(gs_addr + (uint32_t)(s * row_chunks + c) * 16, src + (size_t)c * 16, 16);
+    }
+    ptx::cp_async_commit();
+    ptx::cp_async_wait<0>();
+    __syncthreads();
+
+    const int pairs = dm.C >> 1;
+    const int ti = threadIdx.y;
+    const size_t tokp = (size_t)dm.C;
+    for (int cp0 = 0; cp0 < pairs; cp0 += blockDim.x) {
+        const int cp = cp0 + threadIdx.x;
+        if (cp >= pairs) continue;
+        float2 acc[5], accb = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < 5; ++k) acc[k] = make_float2(0.f, 0.f);
+        for (long long r = r0; r < r1; ++r) {
+            const int y = (int)(r % dm.H);
+            const int yy = y + ti - 2;
+            if (yy < 0 || yy >= dm.H) continue;
+            // 32-bit shared-memory addresses; the window slides along x, five positions per trip so
+            // that the window registers come back to their places without moves
+            const uint32_t tb = (uint32_t)(dm.C * sizeof(T));               // bytes per token
+            uint32_t pg = gs_addr + (uint32_t)(((r - r0) * row_elems + 2 * cp) * sizeof(T));
+            uint32_t pv = vs_addr + (uint32_t)(((r - r0 + ti) * row_elems + 2 * cp) * sizeof(T));
+            float2 w0 = make_float2(0.f, 0.f), w1 = w0;
+            float2 w2 = SmemPair<T>::load(pv);
+            float2 w3 = dm.W > 1 ? SmemPair<T>::load(pv + tb) : make_float2(0.f, 0.f);
+            pv += 2 * tb;
+            int x = 0;
+#define BRA_DW_STEP(WA, WB, WC, WD, WE, G)                 \
+            if (ti == 2) accb = __fadd2_rn(accb, G);        \
+            acc[0] = __ffma2_rn(G, WA, acc[0]);             \
+            acc[1] = __ffma2_rn(G, WB, acc[1]);             \
+            acc[2] = __ffma2_rn(G, WC, acc[2]);             \
+            acc[3] = __ffma2_rn(G, WD, acc[3]);             \
+            acc[4] = __ffma2_rn(G, WE, acc[4]);
+            for (; x + 5 <= dm.W - 2; x += 5) {
+                float2 g[5], nv[5];
+#pragma unroll
+                for (int u = 0; u < 5; ++u) { nv[u] = SmemPair<T>::load(pv + u * tb); g[u] = SmemPair<T>::load(pg + u * tb); }
+                pv += 5 * tb; pg += 5 * tb;
+                BRA_DW_STEP(w0, w1, w2, w3, nv[0], g[0])
+                BRA_DW_STEP(w1, w2, w3, nv[0], nv[1], g[1])
+                BRA_DW_STEP(w2, w3, nv[0], nv[1], nv[2], g[2])
+                BRA_DW_STEP(w3, nv[0], nv[1], nv[2], nv[3], g[3])
+                BRA_DW_STEP(nv[0], nv[1], nv[2], nv[3], nv[4], g[4])
+                w0 = nv[1]; w1 = nv[2]; w2 = nv[3]; w3 = nv[4];
             }
-            __syncthreads();
+            for (; x < dm.W; ++x) {
+                const float2 w4 = x + 2 < dm.W ? SmemPair<T>::load(pv) : make_float2(0.f, 0.f);
+                const float2 g1 = SmemPair<T>::load(pg);
+                pv += tb; pg += tb;
+                BRA_DW_STEP(w0, w1, w2, w3, w4, g1)
+                w0 = w1; w1 = w2; w2 = w3; w3 = w4;
+            }
+#undef BRA_DW_STEP
         }
-        if (threadIdx.y == 0 && active) {
-            float* out = part + ((size_t)blockIdx.x * dm.C + 2 * cp) * 26;
+        float* out = part + ((size_t)blockIdx.x * dm.C + 2 * cp) * 26;
 #pragma unroll
-            for (int k = 0; k < 26; ++k) { out[k] = red[threadIdx.x * 26 + k].x; out[26 + k] = red[threadIdx.x * 26 + k].y; }
-        }
-        __syncthreads();
+        for (int k = 0; k < 5; ++k) { out[ti * 5 + k] = acc[k].x; out[26 + ti * 5 + k] = acc[k].y; }
+        if (ti == 2) { out[25] = accb.x; out[26 + 25] = accb.y; }
     }
 }
 
@@ -377,7 +470,18 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
         const int rpb = (int)((rows + L.dw_blocks - 1) / L.dw_blocks);
         const int nblk = (int)((rows + rpb - 1) / rpb);
         const int cpx = d.C / 2 < DW_CP ? d.C / 2 : DW_CP;
-        bwd_dw_partial_kernel<T><<<nblk, dim3(cpx, DW_SLOTS), sizeof(float2) * cpx * 26, st>>>(v, go, part, rpb, d);
+        const size_t dw_smem = (size_t)(2 * rpb + 4) * d.W * d.C * sizeof(T);
+        if (dw_smem <= 100 * 1024 && ((size_t)d.W * d.C * sizeof(T)) % 16 == 0) {
+            static size_t dw_set = 0;
+            if (dw_smem > 48 * 1024 && dw_smem > dw_set) {
+                if ((e = cudaFuncSetAttribute(bwd_dw_partial_staged_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)dw_smem)) != cudaSuccess) return e;
+                dw_set = dw_smem;
+            }
+            bwd_dw_partial_staged_kernel<T><<<nblk, dim3(cpx, DW_TI), dw_smem, st>>>(v, go, part, rpb, d);
+        } else {
+            bwd_dw_partial_kernel<T><<<nblk, dim3(cpx, DW_TI), 0, st>>>(v, go, part, rpb, d);
+        }
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         bwd_dw_final_kernel<<<(d.C * 26 + 31) / 32, dim3(32, 8), 0, st>>>(part, nblk, d.lce ? d_lce_w : nullptr, d_lce_b, d);
