@@ -15,16 +15,14 @@
 //   3. the warp parks its normalised O^att tile (fp32, warp-private), adds the 5 x 5 depthwise
 //      correlation of V read from the resident V slice (zero outside the map) and stores bf16.
 // No CTA-wide barrier after the set-up: the warps never wait for one another.
-#include "mma_common.cuh"
+#include "img_common.cuh"
 
 namespace bra {
 
 using namespace ptx;
 
 namespace img {
-constexpr int KB = 64;            // keys per block
 constexpr int MAX_WARPS = 8;
-constexpr int MAX_ENTRIES = 8192; // routing entries of one (image, head): R * topk
 }  // namespace img
 
 struct ImgGeom {
@@ -35,76 +33,6 @@ struct ImgGeom {
     uint32_t mul_nr, mul_ws, mul_s, mul_tpr;
     int off_k, off_v, off_idx, off_w, off_st, smem_bytes;
 };
-
-__device__ __forceinline__ uint32_t ldg_u32(const uint8_t* p) {
-    return __ldg(reinterpret_cast<const uint32_t*>(p));
-}
-
-
-// 5 x 5 depthwise correlation (LCE) of the resident V slice for a block of BR rows x WS columns of
-// tokens whose top-left token is (y, x) of the map, for one channel pair: sums added into acc.
-// WS and x are even, so the tokens of a window row pair up on one swizzle phase: one address per
-// pair of loads.  BORDER: the 2-token frame of the block may leave the map (zeros there).
-template <int WS, int BR, bool BORDER>
-__device__ __forceinline__ void lce_block(uint32_t vbase, int y, int x, int H, int W, int cq, uint32_t vcol,
-                                          const float2* wv, float2 (*acc)[WS]) {
-    constexpr int WW = WS + 4;
-#pragma unroll
-    for (int yy = 0; yy < BR + 4; ++yy) {
-        const int iy = y + yy - 2;
-        const bool row_ok = !BORDER || (unsigned)iy < (unsigned)H;
-        const int rt = iy * W + x - 2;                       // token id of the window row's first column
-        float2 v[WW];
-#pragma unroll
-        for (int j = 0; j < WW / 2; ++j) {
-            const int tok = rt + 2 * j;                      // even: tok and tok + 1 share (tok >> 1) & 3
-            const uint32_t a = vbase + tok * 64 + ((cq ^ ((tok >> 1) & 3)) << 4) + vcol;
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int ix = x + 2 * j + e - 2;
-                uint32_t w = 0u;
-                if (row_ok && (!BORDER || (unsigned)ix < (unsigned)W)) w = lds_u32(a + e * 64);
-                v[2 * j + e] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-            }
-        }
-#pragma unroll
-        for (int tj = 0; tj < 5; ++tj)
-#pragma unroll
-            for (int ti = 0; ti < 5; ++ti) {
-                const int r = yy - ti;
-                if (r < 0 || r >= BR) continue;
-#pragma unroll
-                for (int c = 0; c < WS; ++c) acc[r][c] = __ffma2_rn(wv[ti * 5 + tj], v[c + tj], acc[r][c]);
-            }
-    }
-}
-
-// One lane's share of a unit whose 16 (or 4) tokens form full region rows: BR rows x WS columns from
-// row r0 of the tile; adds the parked O^att and stores bf16.
-template <int WS, int BR>
-__device__ __forceinline__ void lce_store_block(uint32_t vbase, const float* stage_o, uint32_t* outb, int r0,
-                                                int y0, int x0, const Dims& dm, int cp, bool lce,
-                                                const float2* wv, float2 bias2) {
-    float2 acc[BR][WS];
-#pragma unroll
-    for (int r = 0; r < BR; ++r)
-#pragma unroll
-        for (int c = 0; c < WS; ++c) acc[r][c] = bias2;
-    const int y = y0 + r0, x = x0;
-    if (lce) {
-        const bool inside = y >= 2 && y + BR + 1 < dm.H && x >= 2 && x + WS + 1 < dm.W;
-        if (inside) lce_block<WS, BR, false>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wv, acc);
-        else        lce_block<WS, BR, true>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wv, acc);
-    }
-#pragma unroll
-    for (int r = 0; r < BR; ++r)
-#pragma unroll
-        for (int c = 0; c < WS; ++c) {
-            const float2 att = *reinterpret_cast<const float2*>(stage_o + ((r0 + r) * WS + c) * 32 + 2 * cp);
-            const float2 r2 = __fadd2_rn(att, acc[r][c]);
-            outb[((size_t)(y + r) * dm.W + x + c) * (dm.C / 2)] = pack2_bf16(r2.x, r2.y);
-        }
-}
 
 // SMALL: CTAs of up to 5 warps (two per SM by shared memory): room for ~200 registers per thread.
 template <bool SMALL>
@@ -129,23 +57,11 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
 
     // ---- 1. the head's K and V slices of the whole image (inputs of the call: no need to wait
     //         for the routing kernel this launch may overlap) ----
-    for (int c = tid; c < dm.N * 4; c += nthreads) {
-        const int tok = c >> 2, q = c & 3;
-        const uint32_t dst = tok * 64 + ((q ^ ((tok >> 1) & 3)) << 4);
-        const size_t src = (size_t)tok * tok_bytes + q * 16;
-        cp_async_16(sbase + gm.off_k + dst, Kb + src, 16);
-        cp_async_16(sbase + gm.off_v + dst, Vb + src, 16);
-    }
+    img_load_slice(sbase + gm.off_k, Kb, dm.N, tok_bytes, tid, nthreads);
+    img_load_slice(sbase + gm.off_v, Vb, dm.N, tok_bytes, tid, nthreads);
     cp_async_commit();
     // LCE weights of the head as [tap][channel pair] (read back conflict-free)
-    if (dm.lce) {
-        const float* wp = lce_w + (size_t)h * 32 * 25;
-        for (int idx = tid; idx < 25 * 16; idx += nthreads) {
-            const int q = idx >> 4, cp = idx & 15;
-            *reinterpret_cast<float2*>(smem + gm.off_w + idx * 8) =
-                make_float2(__ldg(wp + (2 * cp) * 25 + q), __ldg(wp + (2 * cp + 1) * 25 + q));
-        }
-    }
+    if (dm.lce) img_load_weights(smem + gm.off_w, lce_w + (size_t)h * 32 * 25, false, tid, nthreads);
     pdl_wait();          // the index may come from the routing kernel this launch overlaps
     // routing rows of this (image, head): coherent loads, checked once, kept as token ids (-1: bad entry)
     int32_t* s_idx = reinterpret_cast<int32_t*>(smem + gm.off_idx);
@@ -359,60 +275,8 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
         }
         __syncwarp();
 
-        // ---- LCE + store: lane = (channel pair, every other run of `run` tokens along x) ----
-        {
-            float2 wv[25];
-            if (dm.lce) {
-#pragma unroll
-                for (int q = 0; q < 25; ++q) wv[q] = lds_f32x2(sbase + gm.off_w + (q * 16 + cp) * 8);
-            }
-            const uint32_t vcol = (cp & 3) * 4;
-            const int cq = cp >> 2;
-            // the two region shapes of the late stages: whole rows per half-warp, one shared window
-            const bool blk44 = dm.ws == 4 && rows == 16, blk22 = dm.ws == 2 && rows == 4;
-            if (blk44) lce_store_block<4, 2>(vbase, stage_o, outb, 2 * (lane >> 4), y0, x0, dm, cp, dm.lce, wv, bias2);
-            if (blk22) lce_store_block<2, 1>(vbase, stage_o, outb, lane >> 4, y0, x0, dm, cp, dm.lce, wv, bias2);
-            const int nruns = (blk44 || blk22) ? 0 : rows / run;      // tiles start at multiples of 16, n_r is a multiple of run
-            for (int u2 = lane >> 4; u2 < nruns; u2 += 2) {
-                const int t = t0 + u2 * run;
-                const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
-                const int y = y0 + ty, x = x0 + tx;
-                float2 acc[2] = {bias2, bias2};
-                if (dm.lce) {
-                    const bool inside = y >= 2 && y + 2 < dm.H && x >= 2 && x + run + 1 < dm.W;
-#pragma unroll
-                    for (int ti = 0; ti < 5; ++ti) {
-                        const int yy = y + ti - 2;
-                        float2 v[6];
-#pragma unroll
-                        for (int xx = 0; xx < 6; ++xx) {
-                            if (xx < run + 4) {
-                                const int xc = x + xx - 2;
-                                uint32_t w = 0u;
-                                if (inside || ((unsigned)yy < (unsigned)dm.H && (unsigned)xc < (unsigned)dm.W)) {
-                                    const int tok = yy * dm.W + xc;
-                                    w = lds_u32(vbase + tok * 64 + ((cq ^ ((tok >> 1) & 3)) << 4) + vcol);
-                                }
-                                v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-                            }
-                        }
-#pragma unroll
-                        for (int tj = 0; tj < 5; ++tj) {
-                            acc[0] = __ffma2_rn(wv[ti * 5 + tj], v[tj], acc[0]);
-                            if (run == 2) acc[1] = __ffma2_rn(wv[ti * 5 + tj], v[tj + 1], acc[1]);
-                        }
-                    }
-                }
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    if (e < run) {
-                        const float2 att = *reinterpret_cast<const float2*>(stage_o + (t - t0 + e) * 32 + 2 * cp);
-                        const float2 r2 = __fadd2_rn(att, acc[e]);
-                        outb[((size_t)y * dm.W + x + e) * (dm.C / 2)] = pack2_bf16(r2.x, r2.y);
-                    }
-                }
-            }
-        }
+        // ---- LCE + store ----
+        img_lce_store(vbase, dm.lce ? sbase + gm.off_w : 0u, stage_o, outb, t0, rows, y0, x0, dm, gm.mul_ws, lane, bias2);
         __syncwarp();                                                 // the staging tile is read: next unit may overwrite it
     }
 }

@@ -421,6 +421,9 @@ bwd_dw_final_kernel(const float* __restrict__ part, int blocks,
     }
 }
 
+static thread_local int g_bwd_impl = BRA_IMPL_AUTO;
+void hint_backward_impl(int impl) { g_bwd_impl = impl; }
+
 bool backward_supported(const Dims& d) {
     return (d.d == 16 || d.d == 32 || d.d == 64) && d.R <= 1000;
 }
@@ -448,7 +451,15 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-    if (sizeof(T) == 2 && backward_mma_supported(d, BRA_BF16)) {
+    // bf16, head dim 32: tensor-core kernels.  Small maps with enough (image, head) pairs to fill the
+    // GPU keep a whole slice resident; the rest stream blocks through shared memory.
+    const bool img_ok = sizeof(T) == 2 && backward_img_supported(d, BRA_BF16);
+    const bool use_img = img_ok && (g_bwd_impl == BRA_IMPL_IMG ||
+                                    (g_bwd_impl == BRA_IMPL_AUTO && (long long)d.B * d.heads >= 64));
+    if (use_img) {
+        if ((e = launch_backward_img(d, Q, K, V, index, inv_off, inv_list, lce_w, lse, dO, dQ, dK, dV,
+                                     delta, status, st)) != cudaSuccess) return e;
+    } else if (sizeof(T) == 2 && g_bwd_impl != BRA_IMPL_SIMT && backward_mma_supported(d, BRA_BF16)) {
         // head dim 32, bf16: the two tensor-core kernels (dQ + delta, then dK / dV)
         if ((e = launch_backward_mma(d, Q, K, V, index, inv_off, inv_list, lce_w, lse, dO, dQ, dK, dV,
                                      delta, status, st)) != cudaSuccess) return e;

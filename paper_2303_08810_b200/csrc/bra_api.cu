@@ -217,6 +217,7 @@ bra_status bra_backward(const bra_problem* p, const void* Q, const void* K, cons
     WsLayout L;
     if ((s = check_ws(d, ws, ws_bytes, &L)) != BRA_OK) return s;
     if (!backward_supported(d)) return BRA_ERR_UNSUPPORTED;
+    hint_backward_impl(p->impl);
     cudaError_t e = launch_backward(d, p->dtype, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV,
                                     d_lce_w, d_lce_b, static_cast<char*>(ws), L,
                                     static_cast<cudaStream_t>(stream));

@@ -90,6 +90,13 @@ cudaError_t launch_backward_mma(const Dims& d, const void* Q, const void* K, con
                                 const float* lce_w, const float* lse, const void* dO,
                                 void* dQ, void* dK, void* dV, float* delta, int32_t* status, cudaStream_t st);
 
+bool backward_img_supported(const Dims& d, int dtype);
+cudaError_t launch_backward_img(const Dims& d, const void* Q, const void* K, const void* V,
+                                const int32_t* index, const int32_t* inv_off, const int32_t* inv_list,
+                                const float* lce_w, const float* lse, const void* dO,
+                                void* dQ, void* dK, void* dV, float* delta, int32_t* status, cudaStream_t st);
+
+void hint_backward_impl(int impl);     // bra_impl of the call that follows on this thread
 bool backward_supported(const Dims& d);
 cudaError_t launch_backward(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
                             const int32_t* index, const float* lce_w, const float* lse,

@@ -406,11 +406,11 @@ def test_forward_orders_attention_after_routing(bra, n):
 
 
 # ------------------------------------------------------------------ backward
-def run_backward_case(bra, cfg, seed, clustered=False, shared=False, index=None):
+def run_backward_case(bra, cfg, seed, clustered=False, shared=False, index=None, impl="auto"):
     import torch
     x = synthetic.make_inputs(cfg, seed=seed, with_do=True, clustered=clustered)
     t = to_dev(x, cfg)
-    p = problem_of(bra, cfg, shared_routing=shared)
+    p = problem_of(bra, cfg, impl=IMPLS[impl], shared_routing=shared)
     ws = bra.workspace(p)
     if index is None:
         O, idx, lse = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
@@ -453,6 +453,29 @@ BWD_MMA_CASES = [
 @pytest.mark.parametrize("cfg", BWD_MMA_CASES, ids=[c.name for c in BWD_MMA_CASES])
 def test_backward_tensor_core_shapes(bra, cfg):
     run_backward_case(bra, cfg, seed=31)
+
+
+# maps small enough for the kernels that keep a whole (image, head) slice in shared memory
+BWD_IMG_CASES = [c for c in BWD_MMA_CASES if c.H * c.W <= 1500] + [
+    BraConfig("bwd-img-4x4-regions-k4", 3, 28, 28, 128, 4, 7, 4, "bf16"),
+    BraConfig("bwd-img-tail-tile-n_r=24", 2, 12, 16, 64, 2, 2, 3, "bf16"),
+    BraConfig("bwd-img-many-images", 40, 14, 14, 64, 2, 7, 5, "bf16"),
+]
+
+
+@pytest.mark.parametrize("cfg", BWD_IMG_CASES, ids=[c.name for c in BWD_IMG_CASES])
+def test_backward_image_resident_shapes(bra, cfg):
+    run_backward_case(bra, cfg, seed=33, impl="img")
+
+
+def test_backward_image_resident_options(bra):
+    cfg = BraConfig("bwd-img-opts", 2, 16, 16, 64, 2, 4, 3, "bf16")
+    run_backward_case(bra, cfg, seed=34, impl="img", shared=True)
+    run_backward_case(bra, cfg, seed=34, impl="img", clustered=True)
+    idx = np.zeros((cfg.B, cfg.heads, cfg.R, cfg.topk), dtype=np.int32)
+    idx[..., 1] = np.arange(cfg.R)[None, None, :] % 5
+    idx[..., 2] = 3
+    run_backward_case(bra, cfg, seed=35, impl="img", index=idx)
 
 
 def test_backward_tensor_core_duplicates_and_fan_in(bra):
