@@ -35,7 +35,7 @@ struct ImgGeom {
 };
 
 // SMALL: CTAs of up to 5 warps (two per SM by shared memory): room for ~200 registers per thread.
-template <bool SMALL>
+template <bool SMALL, int SHAPE>
 __global__ void __launch_bounds__(SMALL ? 160 : img::MAX_WARPS * 32, 2)
 attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
                   const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
@@ -276,7 +276,7 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
         __syncwarp();
 
         // ---- LCE + store ----
-        img_lce_store(vbase, dm.lce ? sbase + gm.off_w : 0u, stage_o, outb, t0, rows, y0, x0, dm, gm.mul_ws, lane, bias2);
+        img_lce_store<SHAPE>(vbase, dm.lce ? sbase + gm.off_w : 0u, stage_o, outb, t0, rows, y0, x0, dm, gm.mul_ws, lane, bias2);
         __syncwarp();                                                 // the staging tile is read: next unit may overwrite it
     }
 }
@@ -315,15 +315,16 @@ bool attend_img_supported(const Dims& d, int dtype) {
     return img_geom(d, 1).smem_bytes <= 200 * 1024;
 }
 
-template <bool SMALL>
-static cudaError_t img_occupancy(int nw, int smem_bytes, int* occ) {
-    static int smem_set = 0;
-    if (smem_bytes > smem_set) {
-        cudaError_t e = cudaFuncSetAttribute(attend_img_kernel<SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-        if (e != cudaSuccess) return e;
-        smem_set = smem_bytes;
-    }
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, attend_img_kernel<SMALL>, nw * 32, smem_bytes);
+typedef void (*AttendImgKernel)(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*, const int32_t*,
+                                const float*, const float*, __nv_bfloat16*, float*, int32_t*, Dims, ImgGeom);
+static AttendImgKernel img_kernel(bool small, int shape) {
+    if (small) return shape == 44 ? attend_img_kernel<true, 44> : shape == 22 ? attend_img_kernel<true, 22> : attend_img_kernel<true, 0>;
+    return shape == 44 ? attend_img_kernel<false, 44> : shape == 22 ? attend_img_kernel<false, 22> : attend_img_kernel<false, 0>;
+}
+static cudaError_t img_occupancy(AttendImgKernel kernel, int nw, int smem_bytes, int* occ) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, kernel, nw * 32, smem_bytes);
 }
 
 cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
@@ -332,6 +333,7 @@ cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const
     // warps per CTA: the most that still lets every CTA of the grid be resident at once; if no
     // choice does, the one with the most warps per SM.  Remembered per shape.
     const long long grid = (long long)d.B * d.heads;
+    const int shape = img_region_shape(d);
     static thread_local struct { long long grid; int N, ents, nw; } memo = {0, 0, 0, 0};
     int best_nw = 0;
     if (memo.nw && memo.grid == grid && memo.N == d.N && memo.ents == d.R * d.topk) {
@@ -343,8 +345,7 @@ cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const
             const ImgGeom g = img_geom(d, nw);
             if (g.smem_bytes > 200 * 1024) continue;
             int occ = 0;
-            const cudaError_t e = nw <= 5 ? img_occupancy<true>(nw, g.smem_bytes, &occ)
-                                          : img_occupancy<false>(nw, g.smem_bytes, &occ);
+            const cudaError_t e = img_occupancy(img_kernel(nw <= 5, shape), nw, g.smem_bytes, &occ);
             if (e != cudaSuccess) return e;
             if (occ <= 0) continue;
             if ((long long)occ * sms >= grid) { best_nw = nw; break; }
@@ -358,13 +359,11 @@ cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const
     const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(K);
     const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(V);
     const bool pdl = take_after_own_kernel();
-    cudaError_t e;
-    if (best_nw <= 5)
-        e = launch_kernel(attend_img_kernel<true>, dim3((unsigned)grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st, pdl,
-                          q, k, v, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, g);
-    else
-        e = launch_kernel(attend_img_kernel<false>, dim3((unsigned)grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st, pdl,
-                          q, k, v, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, g);
+    AttendImgKernel kernel = img_kernel(best_nw <= 5, shape);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
+    if (e != cudaSuccess) return e;
+    e = launch_kernel(kernel, dim3((unsigned)grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st, pdl,
+                      q, k, v, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, g);
     count_launch();
     return e;
 }

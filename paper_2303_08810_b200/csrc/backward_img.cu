@@ -202,6 +202,7 @@ bwd_dq_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
 }
 
 // ------------------------------------------------------------------ dK, dV
+template <int SHAPE>
 __global__ void __launch_bounds__(bimg::MAX_WARPS * 32, 1)
 bwd_dkv_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
                    const __nv_bfloat16* __restrict__ Vg, const int32_t* __restrict__ inv_off,
@@ -325,7 +326,7 @@ bwd_dkv_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __
         }
         __syncwarp();
         // dV[y, x] += sum_ij w[i, j] dO[y - i + 2, x - j + 2]: the correlation of dO with the flipped filter
-        img_lce_store(gbase, dm.lce ? sbase + gm.off_w : 0u, stage_v, outv, t0, rows, y0, x0, dm, gm.mul_ws, lane,
+        img_lce_store<SHAPE>(gbase, dm.lce ? sbase + gm.off_w : 0u, stage_v, outv, t0, rows, y0, x0, dm, gm.mul_ws, lane,
                       make_float2(0.f, 0.f));
         __syncwarp();
     }
@@ -396,13 +397,15 @@ cudaError_t launch_backward_img(const Dims& d, const void* Q, const void* K, con
                                 const int32_t* index, const int32_t* inv_off, const int32_t* inv_list,
                                 const float* lce_w, const float* lse, const void* dO,
                                 void* dQ, void* dK, void* dV, float* delta, int32_t* status, cudaStream_t st) {
+    const int shape = img_region_shape(d);
+    auto dkv_kernel = shape == 44 ? bwd_dkv_img_kernel<44> : shape == 22 ? bwd_dkv_img_kernel<22> : bwd_dkv_img_kernel<0>;
     static thread_local struct { long long grid; int N, ents, nw_q, nw_kv; } memo = {0, 0, 0, 0, 0};
     const long long grid = (long long)d.B * d.heads;
     cudaError_t e;
     if (!(memo.nw_q && memo.grid == grid && memo.N == d.N && memo.ents == d.R * d.topk)) {
         int nq = 0, nkv = 0;
         if ((e = pick_warps(bwd_dq_img_kernel, d, false, &nq)) != cudaSuccess) return e;
-        if ((e = pick_warps(bwd_dkv_img_kernel, d, true, &nkv)) != cudaSuccess) return e;
+        if ((e = pick_warps(dkv_kernel, d, true, &nkv)) != cudaSuccess) return e;
         memo.grid = grid; memo.N = d.N; memo.ents = d.R * d.topk; memo.nw_q = nq; memo.nw_kv = nkv;
     }
     const BwdImgGeom a = bwd_img_geom(d, memo.nw_q, false), b = bwd_img_geom(d, memo.nw_kv, true);
@@ -414,7 +417,7 @@ cudaError_t launch_backward_img(const Dims& d, const void* Q, const void* K, con
                                                                     delta, status, d, a);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    bwd_dkv_img_kernel<<<(unsigned)grid, b.nw * 32, b.smem_bytes, st>>>(q, k, v, inv_off, inv_list, lse, delta, go, lce_w,
+    dkv_kernel<<<(unsigned)grid, b.nw * 32, b.smem_bytes, st>>>(q, k, v, inv_off, inv_list, lse, delta, go, lce_w,
                                                                      static_cast<__nv_bfloat16*>(dK),
                                                                      static_cast<__nv_bfloat16*>(dV), d, b);
     count_launch();

@@ -111,6 +111,9 @@ __device__ __forceinline__ void lce_store_block(uint32_t vbase, const float* sta
 // table at wtab (shared-memory address; 0: no correlation), for the `rows` tokens from t0 of the
 // region whose first token is (y0, x0); bf16 store of the head's 32 channels.  lane = (channel
 // pair, half): whole region rows per half-warp for 4 x 4 and 2 x 2 regions, else runs along x.
+// SHAPE: 44 = every region is 4 x 4 tokens, 22 = 2 x 2, 0 = anything (decided at launch: each
+// instantiation carries one code path, which keeps the kernels inside the instruction cache).
+template <int SHAPE>
 __device__ __forceinline__ void img_lce_store(uint32_t vbase, uint32_t wtab, const float* stage_o, uint32_t* outb,
                                               int t0, int rows, int y0, int x0, const Dims& dm, uint32_t mul_ws,
                                               int lane, float2 bias2) {
@@ -124,10 +127,9 @@ __device__ __forceinline__ void img_lce_store(uint32_t vbase, uint32_t wtab, con
     const uint32_t vcol = (cp & 3) * 4;
     const int cq = cp >> 2;
     const int run = (dm.ws & 1) ? 1 : 2;
-    const bool blk44 = dm.ws == 4 && rows == 16, blk22 = dm.ws == 2 && rows == 4;
-    if (blk44) lce_store_block<4, 2>(vbase, stage_o, outb, 2 * (lane >> 4), y0, x0, dm, cp, lce, wv, bias2);
-    if (blk22) lce_store_block<2, 1>(vbase, stage_o, outb, lane >> 4, y0, x0, dm, cp, lce, wv, bias2);
-    const int nruns = (blk44 || blk22) ? 0 : rows / run;      // tiles start at multiples of 16, n_r is a multiple of run
+    if (SHAPE == 44) { lce_store_block<4, 2>(vbase, stage_o, outb, 2 * (lane >> 4), y0, x0, dm, cp, lce, wv, bias2); return; }
+    if (SHAPE == 22) { lce_store_block<2, 1>(vbase, stage_o, outb, lane >> 4, y0, x0, dm, cp, lce, wv, bias2); return; }
+    const int nruns = rows / run;                             // tiles start at multiples of 16, n_r is a multiple of run
     for (int u2 = lane >> 4; u2 < nruns; u2 += 2) {
         const int t = t0 + u2 * run;
         const int ty = fdiv(t, dm.ws, mul_ws), tx = t - ty * dm.ws;
@@ -222,6 +224,13 @@ __device__ __forceinline__ void img_load_a_global(uint32_t a[2][4], const uint8_
         a[s][2] = va ? ldg_u32(pa + 32 * s + 16) : 0u;
         a[s][3] = vb ? ldg_u32(pb + 32 * s + 16) : 0u;
     }
+}
+
+// which instantiation a problem takes
+inline int img_region_shape(const Dims& d) {
+    if (d.ws == 4 && d.hs == 4) return 44;
+    if (d.ws == 2 && d.hs == 2) return 22;
+    return 0;
 }
 
 }  // namespace bra
