@@ -443,20 +443,22 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
     const T* v = static_cast<const T*>(V); const T* go = static_cast<const T*>(dO);
     cudaError_t e;
 
-    const int thr = 256;
-    const size_t idx_bytes = sizeof(int32_t) * (size_t)d.R * d.topk;
-    const int staged = idx_bytes <= 40 * 1024;
-    inverse_index_kernel<<<d.B * d.heads_i, thr, sizeof(int32_t) * (d.R + 1) + (staged ? idx_bytes : 0), st>>>(
-        index, inv_off, inv_list, staged, d);
-    count_launch();
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-
     // bf16, head dim 32: tensor-core kernels.  Small maps with enough (image, head) pairs to fill the
     // GPU keep a whole slice resident; the rest stream blocks through shared memory.
     const bool img_ok = sizeof(T) == 2 && backward_img_supported(d, BRA_BF16);
     const bool use_img = img_ok && (g_bwd_impl == BRA_IMPL_IMG ||
                                     (g_bwd_impl == BRA_IMPL_AUTO && (long long)d.B * d.heads >= 64));
+    if (!use_img) {
+        const int thr = 256;
+        const size_t idx_bytes = sizeof(int32_t) * (size_t)d.R * d.topk;
+        const int staged = idx_bytes <= 40 * 1024;
+        inverse_index_kernel<<<d.B * d.heads_i, thr, sizeof(int32_t) * (d.R + 1) + (staged ? idx_bytes : 0), st>>>(
+            index, inv_off, inv_list, staged, d);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
     if (use_img) {
+        // the dQ kernel of this family also writes the inverse routing index
         if ((e = launch_backward_img(d, Q, K, V, index, inv_off, inv_list, lce_w, lse, dO, dQ, dK, dV,
                                      delta, status, st)) != cudaSuccess) return e;
     } else if (sizeof(T) == 2 && g_bwd_impl != BRA_IMPL_SIMT && backward_mma_supported(d, BRA_BF16)) {

@@ -23,7 +23,7 @@ constexpr int MAX_WARPS = 12;
 
 struct BwdImgGeom {
     int nw, tpr, units, nblocks;          // nblocks: key blocks of a query tile (dQ kernel)
-    uint32_t mul_nr, mul_ws, mul_s, mul_tpr;
+    uint32_t mul_nr, mul_ws, mul_s, mul_tpr, mul_k;
     int off_a, off_b;                     // the two resident slices
     int off_idx;                          // dQ: routing rows as token ids; dK/dV: inverse offsets [R + 1], then the lists as token ids
     int off_w, off_st, off_stat, smem_bytes;
@@ -80,6 +80,7 @@ bwd_dq_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
                   const __nv_bfloat16* __restrict__ Vg, const int32_t* __restrict__ index,
                   const float* __restrict__ lse, const __nv_bfloat16* __restrict__ dOg,
                   __nv_bfloat16* __restrict__ dQg, float* __restrict__ delta_out,
+                  int32_t* __restrict__ inv_off, int32_t* __restrict__ inv_list,
                   int32_t* __restrict__ status, Dims dm, BwdImgGeom gm) {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -95,17 +96,57 @@ bwd_dq_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
     img_load_slice(sbase + gm.off_b, reinterpret_cast<const uint8_t*>(Vg) + img_off, dm.N, tok_bytes, tid, nthreads);
     cp_async_commit();
     int32_t* s_idx = reinterpret_cast<int32_t*>(smem + gm.off_idx);
+    int32_t* s_raw = s_idx + dm.R * dm.topk;          // the entries as region numbers (-1: bad entry)
+    int32_t* s_cnt = s_raw + dm.R * dm.topk;          // [R + 1]
+    const int entries = dm.R * dm.topk;
     {
         const int hi = dm.heads_i == 1 ? 0 : h;
         const int32_t* ib = index + ((size_t)b * dm.heads_i + hi) * dm.R * dm.topk;
         for (int e = tid; e < dm.R * dm.topk; e += nthreads) {
             int r = __ldg(ib + e);
             if (r < 0 || r >= dm.R) { record_error(status, BRA_ERR_INDEX, r); r = -1; }
+            s_raw[e] = r;
             if (r >= 0) {
                 const int qy = fdiv(r, dm.S, gm.mul_s), qx = r - qy * dm.S;
                 r = qy * dm.hs * dm.W + qx * dm.ws;
             }
             s_idx[e] = r;
+        }
+    }
+    __syncthreads();
+    // Inverse routing index of this (image, routing head) for the dK / dV kernel, while the slices
+    // are still in flight: per key region j the query regions whose rows list j, in entry order
+    // (query region, then slot) - the fixed order of the dK / dV sums.  Warp w takes regions w, w + nw, ...;
+    // it sweeps the entries 32 at a time and finds its region's hits with a ballot.
+    if (inv_off && (dm.heads_i == dm.heads || h == 0)) {
+        for (int j = warp; j < dm.R; j += gm.nw) {
+            int count = 0;
+            for (int e0 = 0; e0 < entries; e0 += 32) {
+                const int e = e0 + lane;
+                count += __popc(__ballot_sync(0xffffffffu, e < entries && s_raw[e] == j));
+            }
+            if (lane == 0) s_cnt[j] = count;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int run = 0;
+            for (int r = 0; r < dm.R; ++r) { const int c = s_cnt[r]; s_cnt[r] = run; run += c; }
+            s_cnt[dm.R] = run;
+        }
+        __syncthreads();
+        const size_t bh = (size_t)b * dm.heads_i + (dm.heads_i == 1 ? 0 : h);
+        int32_t* off = inv_off + bh * (dm.R + 1);
+        for (int j = tid; j <= dm.R; j += nthreads) off[j] = s_cnt[j];
+        for (int j = warp; j < dm.R; j += gm.nw) {
+            int32_t* outl = inv_list + bh * entries + s_cnt[j];
+            int pos = 0;
+            for (int e0 = 0; e0 < entries; e0 += 32) {
+                const int e = e0 + lane;
+                const bool hit = e < entries && s_raw[e] == j;
+                const unsigned m = __ballot_sync(0xffffffffu, hit);
+                if (hit) outl[pos + __popc(m & ((1u << lane) - 1u))] = fdiv(e, dm.topk, gm.mul_k);
+                pos += __popc(m);
+            }
         }
     }
     cp_async_wait<0>();
@@ -339,14 +380,14 @@ static BwdImgGeom bwd_img_geom(const Dims& d, int nw, bool key_centric) {
     g.tpr = (d.n_r + 15) / 16;
     g.units = d.R * g.tpr;
     g.nblocks = (d.topk * d.n_r + img::KB - 1) / img::KB;
-    g.mul_nr = recip32(d.n_r); g.mul_ws = recip32(d.ws); g.mul_s = recip32(d.S); g.mul_tpr = recip32(g.tpr);
+    g.mul_nr = recip32(d.n_r); g.mul_ws = recip32(d.ws); g.mul_s = recip32(d.S); g.mul_tpr = recip32(g.tpr); g.mul_k = recip32(d.topk);
     int off = 0;
     g.off_a = off;    off += d.N * 64;
     g.off_b = off;    off += d.N * 64;
     g.off_st = off;   off += key_centric ? nw * 2048 : 0;
     g.off_stat = off; off += key_centric ? nw * 512 : 0;
     g.off_w = off;    off += key_centric ? 25 * 16 * 8 : 0;
-    g.off_idx = off;  off += (((d.R * d.topk + (key_centric ? d.R + 1 : 0)) * 4 + 15) / 16) * 16;
+    g.off_idx = off;  off += (((d.R * d.topk * (key_centric ? 1 : 2) + d.R + 1) * 4 + 15) / 16) * 16;
     g.smem_bytes = off;
     return g;
 }
@@ -397,6 +438,7 @@ cudaError_t launch_backward_img(const Dims& d, const void* Q, const void* K, con
                                 const int32_t* index, const int32_t* inv_off, const int32_t* inv_list,
                                 const float* lce_w, const float* lse, const void* dO,
                                 void* dQ, void* dK, void* dV, float* delta, int32_t* status, cudaStream_t st) {
+    // inv_off / inv_list are written by the dQ kernel here (no separate inverse-index launch)
     const int shape = img_region_shape(d);
     auto dkv_kernel = shape == 44 ? bwd_dkv_img_kernel<44> : shape == 22 ? bwd_dkv_img_kernel<22> : bwd_dkv_img_kernel<0>;
     static thread_local struct { long long grid; int N, ents, nw_q, nw_kv; } memo = {0, 0, 0, 0, 0};
@@ -414,7 +456,8 @@ cudaError_t launch_backward_img(const Dims& d, const void* Q, const void* K, con
     const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(V);
     const __nv_bfloat16* go = static_cast<const __nv_bfloat16*>(dO);
     bwd_dq_img_kernel<<<(unsigned)grid, a.nw * 32, a.smem_bytes, st>>>(q, k, v, index, lse, go, static_cast<__nv_bfloat16*>(dQ),
-                                                                    delta, status, d, a);
+                                                                    delta, const_cast<int32_t*>(inv_off),
+                                                                    const_cast<int32_t*>(inv_list), status, d, a);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     dkv_kernel<<<(unsigned)grid, b.nw * 32, b.smem_bytes, st>>>(q, k, v, inv_off, inv_list, lse, delta, go, lce_w,
