@@ -220,6 +220,77 @@ route_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ ind
     }
 }
 
+// Routing with one THREAD per affinity row, for larger k: CTA = (image, routing head, chunk of 64
+// rows).  K^r of the head sits in shared memory (read as broadcasts); the thread forms its R scores
+// (Eq. 4: fp32 FMAs over the channels in increasing order, the same sums as the warp-per-row
+// kernel), parks their order-preserving bits in shared memory and picks the top k by k passes of
+// "largest not yet taken, first one on ties" (Eq. 5).  Per row this is a fraction of the
+// instructions of k warp-wide reductions.  (Four lanes per row, with a quad reduction per rank,
+// measured slower: 28 us against 24 us at 512 image-head pairs, R = 49, k = 16.)
+constexpr int ROUTE_T_ROWS = 64;
+
+template <int DC4>   // channels / 4 of a row of Q^r held in registers (8: head dim 32), or 0: any width
+__global__ void __launch_bounds__(ROUTE_T_ROWS)
+route_rows_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ index, Dims dm) {
+    extern __shared__ float4 kt4[];             // [R][dc + 4] floats, then [R][64] score bits
+    float* ks = reinterpret_cast<float*>(kt4);
+    pdl_launch_dependents();
+    pdl_wait();                                  // the means come from the kernel before
+    const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
+    const int dc = dm.heads_i == 1 ? dm.C : dm.d;
+    const int c0 = dm.heads_i == 1 ? 0 : h * dm.d;
+    const int ld = dc + 4;
+    const int dc4 = dc >> 2;
+    uint32_t* sc = reinterpret_cast<uint32_t*>(ks + (size_t)dm.R * ld) + threadIdx.x;   // this row's scores, stride 64
+    const float* kb = k_mean + (size_t)b * dm.R * dm.C + c0;
+    // coherent loads: the means come from the pooling kernel this one may overlap
+    for (int i = threadIdx.x; i < dm.R * dc4; i += blockDim.x) {
+        const int r = i / dc4, c4 = i - r * dc4;
+        *reinterpret_cast<float4*>(&ks[r * ld + 4 * c4]) = __ldcg(reinterpret_cast<const float4*>(kb + (size_t)r * dm.C) + c4);
+    }
+    __syncthreads();
+    const int i = blockIdx.y * ROUTE_T_ROWS + threadIdx.x;
+    if (i >= dm.R) return;
+    const float4* qrow = reinterpret_cast<const float4*>(q_mean + ((size_t)b * dm.R + i) * dm.C + c0);
+    float4 qreg[DC4 > 0 ? DC4 : 1];
+#pragma unroll
+    for (int c4 = 0; c4 < DC4; ++c4) qreg[c4] = __ldcg(qrow + c4);
+    for (int j = 0; j < dm.R; ++j) {
+        const float4* krow = reinterpret_cast<const float4*>(&ks[j * ld]);
+        float acc = 0.f;
+        if (DC4 > 0) {
+#pragma unroll
+            for (int c4 = 0; c4 < DC4; ++c4) {
+                const float4 k4 = krow[c4];
+                acc = fmaf(qreg[c4].x, k4.x, acc);
+                acc = fmaf(qreg[c4].y, k4.y, acc);
+                acc = fmaf(qreg[c4].z, k4.z, acc);
+                acc = fmaf(qreg[c4].w, k4.w, acc);
+            }
+        } else {
+            for (int c4 = 0; c4 < dc4; ++c4) {
+                const float4 q4 = __ldcg(qrow + c4), k4 = krow[c4];
+                acc = fmaf(q4.x, k4.x, acc);
+                acc = fmaf(q4.y, k4.y, acc);
+                acc = fmaf(q4.z, k4.z, acc);
+                acc = fmaf(q4.w, k4.w, acc);
+            }
+        }
+        sc[j * ROUTE_T_ROWS] = ordered_bits(acc);   // never 0 (NaN is canonical after the + 0): 0 marks "taken"
+    }
+    int32_t* out = index + (((size_t)b * dm.heads_i + h) * dm.R + i) * dm.topk;
+    for (int m = 0; m < dm.topk; ++m) {
+        uint32_t best = 0u;
+        int arg = 0;
+        for (int j = 0; j < dm.R; ++j) {
+            const uint32_t v = sc[j * ROUTE_T_ROWS];
+            if (v > best) { best = v; arg = j; }    // strict: the first of equal scores wins
+        }
+        sc[arg * ROUTE_T_ROWS] = 0u;
+        out[m] = arg;
+    }
+}
+
 static size_t route_smem(const Dims& d) {
     const int dc = d.heads_i == 1 ? d.C : d.d;
     return sizeof(float) * ((size_t)d.R * (dc + 4) + (size_t)ROWS_PER_CTA * dc);
@@ -244,8 +315,34 @@ static cudaError_t launch_route_e(const Dims& d, const float* q_mean, const floa
     return e;
 }
 
+static size_t route_rows_smem(const Dims& d) {
+    const int dc = d.heads_i == 1 ? d.C : d.d;
+    return sizeof(float) * (size_t)d.R * (dc + 4) + sizeof(uint32_t) * (size_t)d.R * ROUTE_T_ROWS;
+}
+
+template <int DC4>
+static cudaError_t launch_route_rows(const Dims& d, const float* q_mean, const float* k_mean,
+                                     int32_t* index, cudaStream_t st) {
+    const size_t smem = route_rows_smem(d);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(route_rows_kernel<DC4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    cudaError_t e = launch_kernel(route_rows_kernel<DC4>, dim3(d.B * d.heads_i, (d.R + ROUTE_T_ROWS - 1) / ROUTE_T_ROWS),
+                                  dim3(ROUTE_T_ROWS), smem, st, /*after_own_kernel=*/true, q_mean, k_mean, index, d);
+    count_launch();
+    return e;
+}
+
 cudaError_t launch_route(const Dims& d, const float* q_mean, const float* k_mean,
                          int32_t* index, cudaStream_t st) {
+    // many winners per row and enough (image, head) pairs to fill the GPU with 64-thread CTAs:
+    // one thread per row
+    if (d.topk > 8 && (long long)d.B * d.heads_i >= 256 && route_rows_smem(d) <= 100 * 1024) {
+        const int dc = d.heads_i == 1 ? d.C : d.d;
+        return dc == 32 ? launch_route_rows<8>(d, q_mean, k_mean, index, st)
+                        : launch_route_rows<0>(d, q_mean, k_mean, index, st);
+    }
     if (d.R <= 32) return launch_route_e<1>(d, q_mean, k_mean, index, st);
     if (d.R <= 64) return launch_route_e<2>(d, q_mean, k_mean, index, st);
     if (d.R <= 128) return launch_route_e<4>(d, q_mean, k_mean, index, st);

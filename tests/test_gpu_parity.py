@@ -118,6 +118,9 @@ def test_route_shared_and_odd_shapes(bra):
         (BraConfig("S=1", 2, 5, 7, 16, 1, 1, 1, "f32"), False),
         (BraConfig("S=16", 1, 32, 32, 32, 1, 16, 12, "bf16"), False),
         (BraConfig("R=100", 1, 20, 30, 64, 2, 10, 7, "f32"), True),
+        # many winners per row and many (image, head) pairs: the thread-per-row routing kernel
+        (BraConfig("k=12-many-pairs", 130, 8, 8, 64, 2, 4, 12, "bf16"), False),
+        (BraConfig("k=9-shared-wide-rows", 256, 6, 6, 48, 3, 3, 9, "bf16"), True),
     ]
     for cfg, shared in cases:
         x = synthetic.make_inputs(cfg, seed=77)
@@ -144,6 +147,12 @@ def test_route_exact_ties_go_to_lower_region(bra):
     K0 = torch.randn_like(K)
     _, _, idx0 = bra.bra_route(p, Q0, K0)
     assert (idx0.cpu().numpy() == np.array([0, 1, 2])).all()
+    # the same through the thread-per-row kernel (k > 8, many image-head pairs)
+    cfg = BraConfig("ties-rows", 256, 8, 8, 32, 1, 4, 10, "f32")
+    p = problem_of(bra, cfg)
+    Q = torch.randn(256, 8, 8, 32, device="cuda")
+    _, _, idx = bra.bra_route(p, Q, torch.ones_like(Q))
+    assert (idx.cpu().numpy() == np.arange(10)).all()
 
 
 # ------------------------------------------------------------------ attention
