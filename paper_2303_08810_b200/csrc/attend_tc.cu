@@ -147,7 +147,6 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     const uint32_t tmem = *tmem_slot;
     TileWalker walk;
     walk.init(blockIdx.x, gridDim.x, dm);
-    pdl_wait();          // everything above overlaps the tail of the kernel before (routing, in bra_forward)
 
     // ---- loader mapping: thread copies 16-byte chunk c of the 128-byte channel row (both
     // heads) of token column tx, in token rows lrow..lrow+3 of a region: a warp covers 512
@@ -244,11 +243,12 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     bool ok = true;
     uint32_t n_s = 0, n_o = 0;              // uses of bar_s / bar_o so far (phase parity)
     TileCoord t = walk.coord();
+    // Q and the V halo are inputs of the call: their copies (and everything above) overlap the tail of
+    // the kernel before (routing, in bra_forward); only the routing index has to wait for it
+    if (my_tiles > 0) load_q_halo(t);
+    pdl_wait();
     int2 ent = read_entries(t, 0);          // entries of the unit whose K/V are being loaded
-    if (my_tiles > 0) {
-        load_q_halo(t);
-        load_kv(t, ent, 0);
-    }
+    if (my_tiles > 0) load_kv(t, ent, 0);
     cp_async_commit();
 
     for (int n = 0; n < my_tiles && ok; ++n) {
