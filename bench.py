@@ -188,7 +188,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma", "tc"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma", "tc", "img"])
     ap.add_argument("--sample-images", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lce", action="store_true", help="attention term only (lce_ksize = 0)")
@@ -218,7 +218,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     bra.load_library()
 
-    impl = {"auto": 0, "simt": 1, "mma": 2, "tc": 3}[args.kernel]
+    impl = {"auto": 0, "simt": 1, "mma": 2, "tc": 3, "img": 4}[args.kernel]
     p = bra.make_problem(cfg.B, cfg.H, cfg.W, cfg.C, cfg.heads, cfg.S, cfg.topk, cfg.dtype, impl=impl,
                          lce=not args.no_lce)
     tdtype = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
