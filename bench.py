@@ -10,7 +10,8 @@ shape the headline metric is quoted on).  Prints ONE JSON line.
   value      queries/s (spatial tokens through the whole forward per second),
              inputs resident in HBM, timed with CUDA events, max over ranks
   e2e        same metric with Q, K, V copied from pinned host memory and O
-             copied back inside the timed region of every step
+             copied back inside the timed region of every step (copies and
+             kernels of neighbouring steps overlap on three streams)
   roofline   dominant kernel (routed attention + LCE): algorithmic bytes of
              one launch / its mean duration from CUDA events, against the
              measured HBM copy bandwidth
@@ -288,26 +289,49 @@ def main():
     attend_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
     assert bra.bra_device_status(ws) == 0
 
-    # end to end: pinned host -> device, forward, device -> host, every step
+    # end to end: pinned host -> device, forward, device -> host, every step.  Three streams and two
+    # sets of device buffers, so that the copies of neighbouring steps overlap the kernels (PCIe moves
+    # both ways at once); every copy of every step is inside the timed region.
     hq, hk, hv = (sets[0][j].cpu().pin_memory() for j in range(3))
-    ho = torch.empty_like(hq).pin_memory()
-    dq, dk, dv, do = (torch.empty_like(sets[0][0]) for _ in range(4))
+    ho = [torch.empty_like(hq).pin_memory() for _ in range(2)]
+    dbuf = [[torch.empty_like(sets[0][0]) for _ in range(4)] for _ in range(2)]     # q, k, v, o
     e2e_steps = max(3, min(args.steps, 20))
+    s_in, s_run, s_out = (torch.cuda.Stream(device=dev) for _ in range(3))
+    ev_in = [torch.cuda.Event() for _ in range(2)]       # inputs of the buffer set have arrived
+    ev_run = [torch.cuda.Event() for _ in range(2)]      # forward on the buffer set is done
+    ev_out = [torch.cuda.Event() for _ in range(2)]      # its result has left the device
 
-    def e2e_step():
-        dq.copy_(hq, non_blocking=True)
-        dk.copy_(hk, non_blocking=True)
-        dv.copy_(hv, non_blocking=True)
-        bra.bra_forward(p, dq, dk, dv, w, None, O=do, index=index, ws=ws, want_lse=False)
-        ho.copy_(do, non_blocking=True)
+    def e2e_step(i):
+        sel = i & 1
+        dq, dk, dv, do = dbuf[sel]
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(ev_run[sel])                 # the forward two steps back has read these buffers
+            dq.copy_(hq, non_blocking=True)
+            dk.copy_(hk, non_blocking=True)
+            dv.copy_(hv, non_blocking=True)
+            ev_in[sel].record(s_in)
+        with torch.cuda.stream(s_run):
+            s_run.wait_event(ev_in[sel])
+            s_run.wait_event(ev_out[sel])                # the result two steps back has been copied out
+            bra.bra_forward(p, dq, dk, dv, w, None, O=do, index=index, ws=ws, want_lse=False)
+            ev_run[sel].record(s_run)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_run[sel])
+            ho[sel].copy_(do, non_blocking=True)
+            ev_out[sel].record(s_out)
 
-    for _ in range(3):
-        e2e_step()
+    torch.cuda.synchronize()
+    for i in range(4):
+        e2e_step(i)
+    torch.cuda.synchronize()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
+    s_in.wait_event(e0); s_run.wait_event(e0); s_out.wait_event(e0)
+    for i in range(e2e_steps):
+        e2e_step(i)
+    cur = torch.cuda.current_stream()
+    cur.wait_stream(s_in); cur.wait_stream(s_run); cur.wait_stream(s_out)
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
