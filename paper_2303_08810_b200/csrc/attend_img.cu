@@ -142,7 +142,8 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
             for (int e = 0; e < 4; ++e) o[n][e] = 0.f;
 
         for (int blk = 0; blk < gm.nblocks; ++blk) {
-            // token (= shared-memory row) of keys blk * 64 + lane and + 32; the other lanes fetch them by shuffle
+            // slice rows (byte offset, swizzle phase in bits 4-5) of keys blk * 64 + lane and + 32; the other lanes
+            // fetch them by shuffle
             int trow[2];
             uint32_t vm[2];
 #pragma unroll
@@ -163,7 +164,7 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
                     }
                     const int base = irow[m];
                     valid = base >= 0;
-                    tr = valid ? base + off : 0;
+                    tr = valid ? img_row_offset(base + off) : 0;
                 }
                 trow[e] = tr;
                 vm[e] = __ballot_sync(0xffffffffu, valid);
@@ -173,12 +174,10 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
             float c[8][4];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
                 uint32_t kb[4];
-                const int tr = __shfl_sync(0xffffffffu, trow[j >> 2], ((8 * j) & 31) + (lane & 7));
-                const int q = lane >> 3;                              // channel chunk of this lane's matrix
-                ldmatrix_x4(kbase + tr * 64 + ((q ^ ((tr >> 1) & 3)) << 4), kb);
-                mma_bf16(c[j], qa[0], kb[0], kb[1]);
+                const int xo = __shfl_sync(0xffffffffu, trow[j >> 2], ((8 * j) & 31) + (lane & 7));
+                ldmatrix_x4(kbase + (xo ^ ((lane >> 3) << 4)), kb);   // lane >> 3: channel chunk of this lane's matrix
+                mma_bf16_zero(c[j], qa[0], kb[0], kb[1]);
                 mma_bf16(c[j], qa[1], kb[2], kb[3]);
             }
             // keys that do not count (padding of the last block, out-of-range entries): -inf
@@ -238,12 +237,11 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
             // O += P V: 4 k-steps of 16 keys x 4 channel tiles of 8
 #pragma unroll
             for (int s = 0; s < 4; ++s) {
-                const int tr = __shfl_sync(0xffffffffu, trow[s >> 1], ((16 * s) & 31) + (lane & 7) + ((lane >> 3) & 1) * 8);
+                const int xo = __shfl_sync(0xffffffffu, trow[s >> 1], ((16 * s) & 31) + (lane & 7) + ((lane >> 3) & 1) * 8);
 #pragma unroll
                 for (int np = 0; np < 2; ++np) {
                     uint32_t vb[4];
-                    const int q = 2 * np + (lane >> 4);
-                    ldmatrix_x4_trans(vbase + tr * 64 + ((q ^ ((tr >> 1) & 3)) << 4), vb);
+                    ldmatrix_x4_trans(vbase + (xo ^ ((2 * np + (lane >> 4)) << 4)), vb);
                     mma_bf16(o[2 * np], pa[s], vb[0], vb[1]);
                     mma_bf16(o[2 * np + 1], pa[s], vb[2], vb[3]);
                 }

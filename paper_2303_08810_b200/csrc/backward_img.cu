@@ -29,7 +29,8 @@ struct BwdImgGeom {
     int off_w, off_st, off_stat, smem_bytes;
 };
 
-// slice row of column lane + 32 e of block blk of a list of region origins (token ids), n_r tokens per entry
+// slice row (img_row_offset) of column lane + 32 e of block blk of a list of region origins (token ids),
+// n_r tokens per entry
 struct ColGeom {
     bool fixed_t; int mstep; int m_of[2], toff[2];
 };
@@ -67,7 +68,7 @@ __device__ __forceinline__ void col_rows(const ColGeom& cg, const Dims& dm, cons
             }
             const int base = list[m];
             valid = base >= 0;
-            tr = valid ? base + off : 0;
+            tr = valid ? img_row_offset(base + off) : 0;
         }
         trow[e] = tr;
         vm[e] = __ballot_sync(0xffffffffu, valid);
@@ -319,8 +320,8 @@ bwd_dkv_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const bool valid = (vm[e] >> lane) & 1u;
-                cl[e] = valid ? __ldg(lse + stat0 + trow[e]) * 1.4426950408889634f : 0.f;
-                cd[e] = valid ? __ldg(delta + stat0 + trow[e]) : 0.f;
+                cl[e] = valid ? __ldg(lse + stat0 + (trow[e] >> 6)) * 1.4426950408889634f : 0.f;   // >> 6: the token
+                cd[e] = valid ? __ldg(delta + stat0 + (trow[e] >> 6)) : 0.f;
             }
             float c[8][4], dp[8][4];
             img_rows_x_gather_t(c, ka, qbase, trow, lane);       // S^T = K Q^T

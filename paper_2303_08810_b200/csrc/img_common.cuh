@@ -172,20 +172,20 @@ __device__ __forceinline__ void img_lce_store(uint32_t vbase, uint32_t wtab, con
 }
 
 
-// ---- MMAs against rows gathered from a resident slice.  trow[e]: the slice row (token) of column
-// lane + 32 e of the current block of 64 columns; the lane that needs another column's row gets it
-// by shuffle.
+// ---- MMAs against rows gathered from a resident slice.  trow[e]: the row of column lane + 32 e of
+// the current block of 64 columns, as its byte offset in the slice with the row's swizzle phase in
+// bits 4-5 (img_row_offset); the lane that needs another column's row gets it by shuffle and only
+// has to xor in its own 16-byte chunk.  Slices start on 64-byte boundaries.
+__device__ __forceinline__ int img_row_offset(int tok) { return tok * 64 + (((tok >> 1) & 3) << 4); }
 // C[16 x 64] = A (16 x 32 channels) * rows^T: column c of C is the dot product with row trow(c)
 __device__ __forceinline__ void img_rows_x_gather_t(float c[8][4], const uint32_t a[2][4], uint32_t slice,
                                                     const int trow[2], int lane) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
         uint32_t b[4];
-        const int tr = __shfl_sync(0xffffffffu, trow[j >> 2], ((8 * j) & 31) + (lane & 7));
-        const int q = lane >> 3;                                  // channel chunk of this lane's matrix
-        ldmatrix_x4(slice + tr * 64 + ((q ^ ((tr >> 1) & 3)) << 4), b);
-        mma_bf16(c[j], a[0], b[0], b[1]);
+        const int xo = __shfl_sync(0xffffffffu, trow[j >> 2], ((8 * j) & 31) + (lane & 7));
+        ldmatrix_x4(slice + (xo ^ ((lane >> 3) << 4)), b);        // lane >> 3: channel chunk of this lane's matrix
+        mma_bf16_zero(c[j], a[0], b[0], b[1]);
         mma_bf16(c[j], a[1], b[2], b[3]);
     }
 }
@@ -194,12 +194,11 @@ __device__ __forceinline__ void img_frag_x_gather(float acc[4][4], const uint32_
                                                   const int trow[2], int lane) {
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        const int tr = __shfl_sync(0xffffffffu, trow[s >> 1], ((16 * s) & 31) + (lane & 7) + ((lane >> 3) & 1) * 8);
+        const int xo = __shfl_sync(0xffffffffu, trow[s >> 1], ((16 * s) & 31) + (lane & 7) + ((lane >> 3) & 1) * 8);
 #pragma unroll
         for (int np = 0; np < 2; ++np) {
             uint32_t b[4];
-            const int q = 2 * np + (lane >> 4);
-            ldmatrix_x4_trans(slice + tr * 64 + ((q ^ ((tr >> 1) & 3)) << 4), b);
+            ldmatrix_x4_trans(slice + (xo ^ ((2 * np + (lane >> 4)) << 4)), b);
             mma_bf16(acc[2 * np], a[s], b[0], b[1]);
             mma_bf16(acc[2 * np + 1], a[s], b[2], b[3]);
         }
