@@ -368,7 +368,7 @@ bwd_dkv_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __
         }
         __syncwarp();
         // dV[y, x] += sum_ij w[i, j] dO[y - i + 2, x - j + 2]: the correlation of dO with the flipped filter
-        img_lce_store<SHAPE>(gbase, dm.lce ? sbase + gm.off_w : 0u, stage_v, outv, t0, rows, y0, x0, dm, gm.mul_ws, lane,
+        img_lce_store<SHAPE, true>(gbase, dm.lce ? sbase + gm.off_w : 0u, stage_v, outv, t0, rows, y0, x0, dm, gm.mul_ws, lane,
                       make_float2(0.f, 0.f));
         __syncwarp();
     }

@@ -81,7 +81,8 @@ __device__ __forceinline__ void lce_block(uint32_t vbase, int y, int x, int H, i
 
 // One lane's share of a unit whose 16 (or 4) tokens form full region rows: BR rows x WS columns from
 // row r0 of the tile; adds the parked O^att and stores bf16.
-template <int WS, int BR>
+// ONE_PATH: only the bounds-checked code (smaller; for kernels that are short of instruction cache).
+template <int WS, int BR, bool ONE_PATH>
 __device__ __forceinline__ void lce_store_block(uint32_t vbase, const float* stage_o, uint32_t* outb, int r0,
                                                 int y0, int x0, const Dims& dm, int cp, bool lce,
                                                 const float2* wv, float2 bias2) {
@@ -93,7 +94,7 @@ __device__ __forceinline__ void lce_store_block(uint32_t vbase, const float* sta
     const int y = y0 + r0, x = x0;
     if (lce) {
         const bool inside = y >= 2 && y + BR + 1 < dm.H && x >= 2 && x + WS + 1 < dm.W;
-        if (inside) lce_block<WS, BR, false>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wv, acc);
+        if (!ONE_PATH && inside) lce_block<WS, BR, false>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wv, acc);
         else        lce_block<WS, BR, true>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wv, acc);
     }
 #pragma unroll
@@ -113,7 +114,7 @@ __device__ __forceinline__ void lce_store_block(uint32_t vbase, const float* sta
 // pair, half): whole region rows per half-warp for 4 x 4 and 2 x 2 regions, else runs along x.
 // SHAPE: 44 = every region is 4 x 4 tokens, 22 = 2 x 2, 0 = anything (decided at launch: each
 // instantiation carries one code path, which keeps the kernels inside the instruction cache).
-template <int SHAPE>
+template <int SHAPE, bool ONE_PATH = false>
 __device__ __forceinline__ void img_lce_store(uint32_t vbase, uint32_t wtab, const float* stage_o, uint32_t* outb,
                                               int t0, int rows, int y0, int x0, const Dims& dm, uint32_t mul_ws,
                                               int lane, float2 bias2) {
@@ -127,8 +128,8 @@ __device__ __forceinline__ void img_lce_store(uint32_t vbase, uint32_t wtab, con
     const uint32_t vcol = (cp & 3) * 4;
     const int cq = cp >> 2;
     const int run = (dm.ws & 1) ? 1 : 2;
-    if (SHAPE == 44) { lce_store_block<4, 2>(vbase, stage_o, outb, 2 * (lane >> 4), y0, x0, dm, cp, lce, wv, bias2); return; }
-    if (SHAPE == 22) { lce_store_block<2, 1>(vbase, stage_o, outb, lane >> 4, y0, x0, dm, cp, lce, wv, bias2); return; }
+    if (SHAPE == 44) { lce_store_block<4, 2, ONE_PATH>(vbase, stage_o, outb, 2 * (lane >> 4), y0, x0, dm, cp, lce, wv, bias2); return; }
+    if (SHAPE == 22) { lce_store_block<2, 1, ONE_PATH>(vbase, stage_o, outb, lane >> 4, y0, x0, dm, cp, lce, wv, bias2); return; }
     const int nruns = rows / run;                             // tiles start at multiples of 16, n_r is a multiple of run
     for (int u2 = lane >> 4; u2 < nruns; u2 += 2) {
         const int t = t0 + u2 * run;
