@@ -194,8 +194,7 @@ bwd_dq_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
             int trow[2]; uint32_t vm[2];
             col_rows(cg, dm, gm, irow, total_keys, blk, lane, trow, vm);
             float c[8][4], dp[8][4];
-            img_rows_x_gather_t(c, qa, kbase, trow, lane);      // S = Q K^T
-            img_rows_x_gather_t(dp, ga, vbase, trow, lane);     // dP = dO V^T
+            img_rows_x_gather_t2(c, qa, kbase, dp, ga, vbase, trow, lane);   // S = Q K^T, dP = dO V^T
             // P = exp(S scale - lse); keys that do not count give 0
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -324,8 +323,7 @@ bwd_dkv_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __
                 cd[e] = valid ? __ldg(delta + stat0 + (trow[e] >> 6)) : 0.f;
             }
             float c[8][4], dp[8][4];
-            img_rows_x_gather_t(c, ka, qbase, trow, lane);       // S^T = K Q^T
-            img_rows_x_gather_t(dp, va, gbase, trow, lane);      // dP^T = V dO^T
+            img_rows_x_gather_t2(c, ka, qbase, dp, va, gbase, trow, lane);   // S^T = K Q^T, dP^T = V dO^T
 #pragma unroll
             for (int e = 0; e < 2; ++e) { st[lane + 32 * e] = cl[e]; st[64 + lane + 32 * e] = cd[e]; }
             __syncwarp();
@@ -346,8 +344,7 @@ bwd_dkv_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __
                 sa[j >> 1][(j & 1) * 2] = pack2_bf16(p0 * (dp[j][0] - dl.x), p1 * (dp[j][1] - dl.y));
                 sa[j >> 1][(j & 1) * 2 + 1] = pack2_bf16(p2 * (dp[j][2] - dl.x), p3 * (dp[j][3] - dl.y));
             }
-            img_frag_x_gather(dk, sa, qbase, trow, lane);        // dK += dS^T Q
-            img_frag_x_gather(dv, pa, gbase, trow, lane);        // dV += P^T dO
+            img_frag_x_gather2(dk, sa, qbase, dv, pa, gbase, trow, lane);    // dK += dS^T Q, dV += P^T dO
             __syncwarp();                                        // the statistics may be overwritten
         }
 

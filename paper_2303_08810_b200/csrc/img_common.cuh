@@ -205,6 +205,42 @@ __device__ __forceinline__ void img_frag_x_gather(float acc[4][4], const uint32_
         }
     }
 }
+// The same two products against the rows of TWO slices that share their row numbers (K and V, or Q
+// and dO): one shuffle and one address per pair of loads.
+__device__ __forceinline__ void img_rows_x_gather_t2(float c1[8][4], const uint32_t a1[2][4], uint32_t slice1,
+                                                     float c2[8][4], const uint32_t a2[2][4], uint32_t slice2,
+                                                     const int trow[2], int lane) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        uint32_t b[4];
+        const int xo = __shfl_sync(0xffffffffu, trow[j >> 2], ((8 * j) & 31) + (lane & 7)) ^ ((lane >> 3) << 4);
+        ldmatrix_x4(slice1 + xo, b);
+        mma_bf16_zero(c1[j], a1[0], b[0], b[1]);
+        mma_bf16(c1[j], a1[1], b[2], b[3]);
+        ldmatrix_x4(slice2 + xo, b);
+        mma_bf16_zero(c2[j], a2[0], b[0], b[1]);
+        mma_bf16(c2[j], a2[1], b[2], b[3]);
+    }
+}
+__device__ __forceinline__ void img_frag_x_gather2(float acc1[4][4], const uint32_t a1[4][4], uint32_t slice1,
+                                                   float acc2[4][4], const uint32_t a2[4][4], uint32_t slice2,
+                                                   const int trow[2], int lane) {
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        const int xo = __shfl_sync(0xffffffffu, trow[s >> 1], ((16 * s) & 31) + (lane & 7) + ((lane >> 3) & 1) * 8);
+#pragma unroll
+        for (int np = 0; np < 2; ++np) {
+            uint32_t b[4];
+            const int xq = xo ^ ((2 * np + (lane >> 4)) << 4);
+            ldmatrix_x4_trans(slice1 + xq, b);
+            mma_bf16(acc1[2 * np], a1[s], b[0], b[1]);
+            mma_bf16(acc1[2 * np + 1], a1[s], b[2], b[3]);
+            ldmatrix_x4_trans(slice2 + xq, b);
+            mma_bf16(acc2[2 * np], a2[s], b[0], b[1]);
+            mma_bf16(acc2[2 * np + 1], a2[s], b[2], b[3]);
+        }
+    }
+}
 // A fragments (rows g and g + 8 of a 16-token tile of a region, 32 channels) straight from global
 // memory; rows beyond `rows` are zero.  base: the image's first token, offset to the head.
 __device__ __forceinline__ void img_load_a_global(uint32_t a[2][4], const uint8_t* base, int y0, int x0, int t0,
