@@ -318,11 +318,10 @@ cudaError_t launch_attend_mma(const Dims& d, const void* Q, const void* K, const
                               const int32_t* index, const float* lce_w, const float* lce_b,
                               void* O, float* lse, int32_t* status, cudaStream_t st) {
     const MmaGeom g = mma_geom(d);
-    static int smem_set = 0;
-    if (g.smem_bytes > 48 * 1024 && g.smem_bytes > smem_set) {
+    static PerDeviceMax smem_set;
+    if (g.smem_bytes > 48 * 1024 && smem_set.raise(g.smem_bytes)) {
         cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
         if (e != cudaSuccess) return e;
-        smem_set = g.smem_bytes;
     }
     const unsigned grid = (unsigned)((long long)d.B * d.R * d.heads * g.chunks);
     cudaError_t e = launch_kernel(attend_mma_kernel, dim3(grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st,

@@ -473,8 +473,8 @@ bool attend_tc_supported(const Dims& d, int dtype) {
 cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const void* V,
                              const int32_t* index, const float* lce_w, const float* lce_b,
                              void* O, float* lse, int32_t* status, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceMax attr_set;
+    if (attr_set.raise(1)) {
         cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_K1);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(attend_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_KN);
@@ -484,7 +484,6 @@ cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const 
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(attend_tc_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
-        attr_set = true;
 #ifdef BRA_TRACE
         int occ1 = 0, occn = 0;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ1, attend_tc_kernel<true>, tc::THREADS, tc::SMEM_K1);

@@ -327,13 +327,12 @@ bool attend_tc_wide_supported(const Dims& d, int dtype) {
 cudaError_t launch_attend_tc_wide(const Dims& d, const void* Q, const void* K, const void* V,
                                   const int32_t* index, const float* lce_w, const float* lce_b,
                                   void* O, float* lse, int32_t* status, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceMax attr_set;
+    if (attr_set.raise(1)) {
         cudaError_t e = cudaFuncSetAttribute(attend_tc_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tw::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(attend_tc_wide_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     int dev = 0, sms = 1;
     if (cudaGetDevice(&dev) != cudaSuccess ||

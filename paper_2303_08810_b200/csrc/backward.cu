@@ -485,11 +485,10 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
         const int cpx = d.C / 2 < DW_CP ? d.C / 2 : DW_CP;
         const size_t dw_smem = (size_t)(2 * rpb + 4) * d.W * d.C * sizeof(T);
         if (dw_smem <= 100 * 1024 && ((size_t)d.W * d.C * sizeof(T)) % 16 == 0) {
-            static size_t dw_set = 0;
-            if (dw_smem > 48 * 1024 && dw_smem > dw_set) {
+            static PerDeviceMax dw_set;
+            if (dw_smem > 48 * 1024 && dw_set.raise((int)dw_smem)) {
                 if ((e = cudaFuncSetAttribute(bwd_dw_partial_staged_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)dw_smem)) != cudaSuccess) return e;
-                dw_set = dw_smem;
             }
             bwd_dw_partial_staged_kernel<T><<<nblk, dim3(cpx, DW_TI), dw_smem, st>>>(v, go, part, rpb, d);
         } else {

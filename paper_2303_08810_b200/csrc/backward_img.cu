@@ -439,14 +439,16 @@ cudaError_t launch_backward_img(const Dims& d, const void* Q, const void* K, con
     // inv_off / inv_list are written by the dQ kernel here (no separate inverse-index launch)
     const int shape = img_region_shape(d);
     auto dkv_kernel = shape == 44 ? bwd_dkv_img_kernel<44> : shape == 22 ? bwd_dkv_img_kernel<22> : bwd_dkv_img_kernel<0>;
-    static thread_local struct { long long grid; int N, ents, nw_q, nw_kv; } memo = {0, 0, 0, 0, 0};
+    static thread_local struct { long long grid; int N, ents, dev, nw_q, nw_kv; } memo = {0, 0, 0, -1, 0, 0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorUnknown;
     const long long grid = (long long)d.B * d.heads;
     cudaError_t e;
-    if (!(memo.nw_q && memo.grid == grid && memo.N == d.N && memo.ents == d.R * d.topk)) {
+    if (!(memo.nw_q && memo.grid == grid && memo.N == d.N && memo.ents == d.R * d.topk && memo.dev == dev)) {   // attributes are per device
         int nq = 0, nkv = 0;
         if ((e = pick_warps(bwd_dq_img_kernel, d, false, &nq)) != cudaSuccess) return e;
         if ((e = pick_warps(dkv_kernel, d, true, &nkv)) != cudaSuccess) return e;
-        memo.grid = grid; memo.N = d.N; memo.ents = d.R * d.topk; memo.nw_q = nq; memo.nw_kv = nkv;
+        memo.grid = grid; memo.N = d.N; memo.ents = d.R * d.topk; memo.dev = dev; memo.nw_q = nq; memo.nw_kv = nkv;
     }
     const BwdImgGeom a = bwd_img_geom(d, memo.nw_q, false), b = bwd_img_geom(d, memo.nw_kv, true);
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(Q);

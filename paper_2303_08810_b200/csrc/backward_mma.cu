@@ -477,15 +477,13 @@ cudaError_t launch_backward_mma(const Dims& d, const void* Q, const void* K, con
                                 const float* lce_w, const float* lse, const void* dO,
                                 void* dQ, void* dK, void* dV, float* delta, int32_t* status, cudaStream_t st) {
     const BwdGeom a = bwd_geom(d, false), b = bwd_geom(d, true);
-    static int smem_a = 0, smem_b = 0;
+    static PerDeviceMax smem_a, smem_b;
     cudaError_t e;
-    if (a.smem_bytes > 48 * 1024 && a.smem_bytes > smem_a) {
+    if (a.smem_bytes > 48 * 1024 && smem_a.raise(a.smem_bytes)) {
         if ((e = cudaFuncSetAttribute(bwd_dq_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, a.smem_bytes)) != cudaSuccess) return e;
-        smem_a = a.smem_bytes;
     }
-    if (b.smem_bytes > 48 * 1024 && b.smem_bytes > smem_b) {
+    if (b.smem_bytes > 48 * 1024 && smem_b.raise(b.smem_bytes)) {
         if ((e = cudaFuncSetAttribute(bwd_dkv_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, b.smem_bytes)) != cudaSuccess) return e;
-        smem_b = b.smem_bytes;
     }
     const unsigned grid = (unsigned)((long long)d.B * d.R * d.heads * a.g.chunks);
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(Q);

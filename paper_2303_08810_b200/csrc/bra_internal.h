@@ -96,6 +96,20 @@ cudaError_t launch_backward_img(const Dims& d, const void* Q, const void* K, con
                                 const float* lce_w, const float* lse, const void* dO,
                                 void* dQ, void* dK, void* dV, float* delta, int32_t* status, cudaStream_t st);
 
+// A process may drive several GPUs, and kernel attributes are per device: the largest value already
+// set for a kernel on the CURRENT device (dynamic shared-memory size, or 1 for "set-up done").
+struct PerDeviceMax {
+    int v[64] = {};
+    // true if `want` exceeds what the current device has been given so far; records it
+    bool raise(int want) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+        if (want <= v[dev]) return false;
+        v[dev] = want;
+        return true;
+    }
+};
+
 void hint_backward_impl(int impl);     // bra_impl of the call that follows on this thread
 bool backward_supported(const Dims& d);
 cudaError_t launch_backward(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
