@@ -70,6 +70,7 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int RB = dm.hs / RT;                       // row blocks per region
     const int units = dm.topk * RB;                  // key blocks per tile
+    const int inv_s = (1 << 20) / dm.S + 1;          // r / S == (r * inv_s) >> 20 for r < 4096
 
     if (tid == 0) {
         mbar_init(bar_s, 1);
@@ -99,11 +100,6 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
     // ---- LCE mapping: channel pair cp, two columns, all 8 rows of the tile
     const int cp = lane & 15;
     const int xl0 = 2 * (warp * 2 + (lane >> 4));
-    float2 wv[25];
-#pragma unroll
-    for (int q = 0; q < 25; ++q) wv[q] = make_float2(0.f, 0.f);
-    float2 bias2 = make_float2(0.f, 0.f);
-    int h_loaded = -1;
 
     constexpr uint32_t IDESC_S = umma_idesc_bf16(128, 128, false, false);
     constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 32, false, true);
@@ -125,19 +121,14 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
         const int hi = dm.heads_i == 1 ? 0 : h;
         const int32_t* irow = index + (((size_t)b * dm.heads_i + hi) * dm.R + i) * dm.topk;
 
-        if (dm.lce && h != h_loaded) {
-            const float* wp = lce_w + (size_t)(h * 32 + 2 * cp) * 25;
-#pragma unroll
-            for (int q = 0; q < 25; ++q) wv[q] = make_float2(__ldg(wp + q), __ldg(wp + 25 + q));
-            if (lce_b) bias2 = make_float2(__ldg(lce_b + h * 32 + 2 * cp), __ldg(lce_b + h * 32 + 2 * cp + 1));
-            h_loaded = h;
-        }
         // key block u = (routed slot m, row block of that region); entry -1: out of range, its P is zero
-        auto load_unit = [&](int u, int buf) -> bool {
-            int r = __ldcg(irow + u / RB);   // coherent load: the index may come from the kernel this one overlaps
+        // (u = m * RB + kb: the launcher keeps R <= 4096, so r / S is a multiply and a shift)
+        auto load_unit = [&](int m, int kb, int buf) -> bool {
+            int r = __ldcg(irow + m);        // coherent load: the index may come from the kernel this one overlaps
             const bool valid = r >= 0 && r < dm.R;
             if (!valid) { record_error(status, BRA_ERR_INDEX, r); r = 0; }
-            const size_t off = (size_t)((r / dm.S) * dm.hs + (u % RB) * RT) * row_bytes + (size_t)((r % dm.S) * WS) * tok_bytes;
+            const int qy = (r * inv_s) >> 20, qx = r - qy * dm.S;
+            const size_t off = (size_t)(qy * dm.hs + kb * RT) * row_bytes + (size_t)(qx * WS) * tok_bytes;
             load_block(sm_base + OFF_KV + buf * 16384, Kb + off);
             load_block(sm_base + OFF_KV + buf * 16384 + 8192, Vb + off);
             return valid;
@@ -157,7 +148,8 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
                 }
             }
         }
-        bool valid_next = load_unit(0, 0);
+        bool valid_next = load_unit(0, 0, 0);
+        int m_next = 0, kb_next = 0;             // (routed slot, row block) of the key block being loaded
         cp_async_commit();
 
         float m_run = -INFINITY, l_run = 0.f;
@@ -181,7 +173,8 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
                 umma_commit(bar_s);
             }
             if (u + 1 < units) {                     // next block into the other buffer (its MMAs are done)
-                valid_next = load_unit(u + 1, buf ^ 1);
+                if (++kb_next == RB) { kb_next = 0; ++m_next; }
+                valid_next = load_unit(m_next, kb_next, buf ^ 1);
                 cp_async_commit();
             }
             if (warp == 0) ok = mbar_wait(bar_s, n_mma & 1, POLL_LIMIT);
@@ -208,19 +201,27 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
             // pass 2: P = exp2(S * scale * log2 e - max), bf16 pairs over the consumed columns of S; row sum
             const float2 sl2v = make_float2(sl2, sl2), mnegv = make_float2(mneg, mneg);
             float2 sum2 = make_float2(0.f, 0.f);
+            if (valid) {
 #pragma unroll 1
-            for (int cc = 0; cc < 128; cc += 16) {
-                uint32_t r[16], pk[8];
-                tmem_ld_32x32b_x16(tg + cc, r);
-                tmem_ld_wait();
+                for (int cc = 0; cc < 128; cc += 16) {
+                    uint32_t r[16], pk[8];
+                    tmem_ld_32x32b_x16(tg + cc, r);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int q = 0; q < 16; q += 2) {
-                    const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[q]), __uint_as_float(r[q + 1])), sl2v, mnegv);
-                    const float2 pe = make_float2(valid ? ex2w(a.x) : 0.f, valid ? ex2w(a.y) : 0.f);
-                    sum2 = __fadd2_rn(sum2, pe);
-                    pk[q >> 1] = packw(pe.x, pe.y);
+                    for (int q = 0; q < 16; q += 2) {
+                        const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[q]), __uint_as_float(r[q + 1])), sl2v, mnegv);
+                        const float2 pe = make_float2(ex2w(a.x), ex2w(a.y));
+                        sum2 = __fadd2_rn(sum2, pe);
+                        pk[q >> 1] = packw(pe.x, pe.y);
+                    }
+                    tmem_st_32x32b_x8(tg + (cc >> 1), pk);
                 }
-                tmem_st_32x32b_x8(tg + (cc >> 1), pk);
+            } else {                                 // a bad routing entry (the whole CTA sees it): P = 0
+                uint32_t pk[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) pk[q] = 0u;
+#pragma unroll 1
+                for (int cc = 0; cc < 64; cc += 8) tmem_st_32x32b_x8(tg + cc, pk);
             }
             tmem_st_wait();
             tc_fence_before_sync();
@@ -247,6 +248,16 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
         }
         if (!ok) break;
 
+        // the head's LCE weights for this thread's channel pair: fetched here, not held through the key
+        // loop (50 registers); the loads fly during the staging below
+        float2 wv[25];
+        float2 bias2 = make_float2(0.f, 0.f);
+        if (dm.lce) {
+            const float* wp = lce_w + (size_t)(h * 32 + 2 * cp) * 25;
+#pragma unroll
+            for (int q = 0; q < 25; ++q) wv[q] = make_float2(__ldg(wp + q), __ldg(wp + 25 + q));
+        }
+        if (lce_b) bias2 = make_float2(__ldg(lce_b + h * 32 + 2 * cp), __ldg(lce_b + h * 32 + 2 * cp + 1));
         // ---- normalise, stage O^att as fp32 [128 tokens][32 ch] (16-byte units xor-swizzled) ----
         {
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
@@ -320,7 +331,7 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
 
 // ------------------------------------------------------------------ host side
 bool attend_tc_wide_supported(const Dims& d, int dtype) {
-    return dtype == BRA_BF16 && d.d == 32 && d.ws == tw::WS && d.hs % tw::RT == 0 && d.topk <= tw::KCAP &&
+    return dtype == BRA_BF16 && d.d == 32 && d.ws == tw::WS && d.hs % tw::RT == 0 && d.topk <= tw::KCAP && d.R <= 4096 &&
            (long long)d.B * d.R * d.heads * (d.hs / tw::RT) < (1ll << 30);
 }
 
