@@ -117,36 +117,69 @@ bwd_dq_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
     __syncthreads();
     // Inverse routing index of this (image, routing head) for the dK / dV kernel, while the slices
     // are still in flight: per key region j the query regions whose rows list j, in entry order
-    // (query region, then slot) - the fixed order of the dK / dV sums.  Warp w takes regions w, w + nw, ...;
-    // it sweeps the entries 32 at a time and finds its region's hits with a ballot.
+    // (query region, then slot) - the fixed order of the dK / dV sums.  Counting by comparison: every
+    // thread scans the (few hundred to few thousand) entries in shared memory on its own.
     if (inv_off && (dm.heads_i == dm.heads || h == 0)) {
-        for (int j = warp; j < dm.R; j += gm.nw) {
-            int count = 0;
-            for (int e0 = 0; e0 < entries; e0 += 32) {
-                const int e = e0 + lane;
-                count += __popc(__ballot_sync(0xffffffffu, e < entries && s_raw[e] == j));
+        const bool by_scan = entries <= 1024;       // few entries: every thread scans them on its own
+        // how many entries name region j
+        if (by_scan) {
+            for (int j = tid; j < dm.R; j += nthreads) {
+                int count = 0;
+                for (int e = 0; e < entries; ++e) count += s_raw[e] == j;
+                s_cnt[j] = count;
             }
-            if (lane == 0) s_cnt[j] = count;
+        } else {                                    // many: a warp per region, 32 entries at a time, ballots
+            for (int j = warp; j < dm.R; j += gm.nw) {
+                int count = 0;
+                for (int e0 = 0; e0 < entries; e0 += 32) {
+                    const int e = e0 + lane;
+                    count += __popc(__ballot_sync(0xffffffffu, e < entries && s_raw[e] == j));
+                }
+                if (lane == 0) s_cnt[j] = count;
+            }
         }
         __syncthreads();
-        if (tid == 0) {
-            int run = 0;
-            for (int r = 0; r < dm.R; ++r) { const int c = s_cnt[r]; s_cnt[r] = run; run += c; }
-            s_cnt[dm.R] = run;
+        // exclusive prefix over the regions: one warp, a run of regions per lane
+        if (warp == 0) {
+            const int per = (dm.R + 31) / 32;
+            const int j0 = min(lane * per, dm.R), j1 = min(j0 + per, dm.R);
+            int sum = 0;
+            for (int j = j0; j < j1; ++j) sum += s_cnt[j];
+            int incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            int run = incl - sum;
+            for (int j = j0; j < j1; ++j) { const int c = s_cnt[j]; s_cnt[j] = run; run += c; }
+            if (lane == 31) s_cnt[dm.R] = incl;
         }
         __syncthreads();
         const size_t bh = (size_t)b * dm.heads_i + (dm.heads_i == 1 ? 0 : h);
         int32_t* off = inv_off + bh * (dm.R + 1);
         for (int j = tid; j <= dm.R; j += nthreads) off[j] = s_cnt[j];
-        for (int j = warp; j < dm.R; j += gm.nw) {
-            int32_t* outl = inv_list + bh * entries + s_cnt[j];
-            int pos = 0;
-            for (int e0 = 0; e0 < entries; e0 += 32) {
-                const int e = e0 + lane;
-                const bool hit = e < entries && s_raw[e] == j;
-                const unsigned m = __ballot_sync(0xffffffffu, hit);
-                if (hit) outl[pos + __popc(m & ((1u << lane) - 1u))] = fdiv(e, dm.topk, gm.mul_k);
-                pos += __popc(m);
+        // entry e goes to its region's list at the number of earlier entries that name the same region
+        int32_t* outl = inv_list + bh * entries;
+        if (by_scan) {
+            for (int e = tid; e < entries; e += nthreads) {
+                const int r = s_raw[e];
+                if (r < 0) continue;
+                int rank = 0;
+                for (int e2 = 0; e2 < e; ++e2) rank += s_raw[e2] == r;
+                outl[s_cnt[r] + rank] = fdiv(e, dm.topk, gm.mul_k);
+            }
+        } else {
+            for (int j = warp; j < dm.R; j += gm.nw) {
+                int32_t* lj = outl + s_cnt[j];
+                int pos = 0;
+                for (int e0 = 0; e0 < entries; e0 += 32) {
+                    const int e = e0 + lane;
+                    const bool hit = e < entries && s_raw[e] == j;
+                    const unsigned m = __ballot_sync(0xffffffffu, hit);
+                    if (hit) lj[pos + __popc(m & ((1u << lane) - 1u))] = fdiv(e, dm.topk, gm.mul_k);
+                    pos += __popc(m);
+                }
             }
         }
     }
