@@ -328,36 +328,45 @@ static cudaError_t img_occupancy(AttendImgKernel kernel, int nw, int smem_bytes,
 cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
                               const int32_t* index, const float* lce_w, const float* lce_b,
                               void* O, float* lse, int32_t* status, cudaStream_t st) {
-    // warps per CTA: the most that still lets every CTA of the grid be resident at once; if no
-    // choice does, the one with the most warps per SM.  Remembered per shape.
+    // Warps per CTA and register variant (SMALL: up to ~200 registers, CTAs of at most 5 warps): among
+    // the choices that let every CTA of the grid be resident at once, the one with the most warps per
+    // SM (the roomier variant on a tie); if none does, the most warps per SM.  Remembered per shape.
     const long long grid = (long long)d.B * d.heads;
     const int shape = img_region_shape(d);
-    static thread_local struct { long long grid; int N, ents, nw; } memo = {0, 0, 0, 0};
+    static thread_local struct { long long grid; int N, ents, nw; bool small; } memo = {0, 0, 0, 0, false};
     int best_nw = 0;
+    bool best_small = false;
     if (memo.nw && memo.grid == grid && memo.N == d.N && memo.ents == d.R * d.topk) {
         best_nw = memo.nw;
+        best_small = memo.small;
     } else {
         const int sms = img_sm_count();
         int best_warps = -1;
+        bool best_fits = false;
         for (int nw = img::MAX_WARPS; nw >= 1; --nw) {
             const ImgGeom g = img_geom(d, nw);
             if (g.smem_bytes > 200 * 1024) continue;
-            int occ = 0;
-            const cudaError_t e = img_occupancy(img_kernel(nw <= 5, shape), nw, g.smem_bytes, &occ);
-            if (e != cudaSuccess) return e;
-            if (occ <= 0) continue;
-            if ((long long)occ * sms >= grid) { best_nw = nw; break; }
-            if (occ * nw > best_warps) { best_warps = occ * nw; best_nw = nw; }
+            for (int small = 0; small <= (nw <= 5 ? 1 : 0); ++small) {
+                int occ = 0;
+                const cudaError_t e = img_occupancy(img_kernel(small != 0, shape), nw, g.smem_bytes, &occ);
+                if (e != cudaSuccess) return e;
+                if (occ <= 0) continue;
+                const bool fits = (long long)occ * sms >= grid;
+                const int warps = occ * nw;
+                if ((fits && !best_fits) || (fits == best_fits && warps >= best_warps)) {
+                    best_fits = fits; best_warps = warps; best_nw = nw; best_small = small != 0;
+                }
+            }
         }
         if (!best_nw) return cudaErrorInvalidConfiguration;
-        memo.grid = grid; memo.N = d.N; memo.ents = d.R * d.topk; memo.nw = best_nw;
+        memo.grid = grid; memo.N = d.N; memo.ents = d.R * d.topk; memo.nw = best_nw; memo.small = best_small;
     }
     const ImgGeom g = img_geom(d, best_nw);
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(Q);
     const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(K);
     const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(V);
     const bool pdl = take_after_own_kernel();
-    AttendImgKernel kernel = img_kernel(best_nw <= 5, shape);
+    AttendImgKernel kernel = img_kernel(best_small, shape);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
     if (e != cudaSuccess) return e;
     e = launch_kernel(kernel, dim3((unsigned)grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st, pdl,

@@ -47,7 +47,7 @@ __device__ __forceinline__ uint32_t ldg_u32(const uint8_t* p) {
 // pair of loads.  BORDER: the 2-token frame of the block may leave the map (zeros there).
 template <int WS, int BR, bool BORDER>
 __device__ __forceinline__ void lce_block(uint32_t vbase, int y, int x, int H, int W, int cq, uint32_t vcol,
-                                          const float2* wv, float2 (*acc)[WS]) {
+                                          uint32_t wlane, float2 (*acc)[WS]) {
     constexpr int WW = WS + 4;
 #pragma unroll
     for (int yy = 0; yy < BR + 4; ++yy) {
@@ -67,15 +67,20 @@ __device__ __forceinline__ void lce_block(uint32_t vbase, int y, int x, int H, i
                 v[2 * j + e] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
             }
         }
+        // window row yy meets tap rows ti = yy - r of the block's rows r: their weights come from the table
+        // (wlane: this lane's channel pair) when they are needed, not held in registers throughout
 #pragma unroll
-        for (int tj = 0; tj < 5; ++tj)
+        for (int ti = 0; ti < 5; ++ti) {
+            const int r = yy - ti;
+            if (r < 0 || r >= BR) continue;
+            float2 w[5];
 #pragma unroll
-            for (int ti = 0; ti < 5; ++ti) {
-                const int r = yy - ti;
-                if (r < 0 || r >= BR) continue;
+            for (int tj = 0; tj < 5; ++tj) w[tj] = ptx::lds_f32x2(wlane + (ti * 5 + tj) * 128);
 #pragma unroll
-                for (int c = 0; c < WS; ++c) acc[r][c] = __ffma2_rn(wv[ti * 5 + tj], v[c + tj], acc[r][c]);
-            }
+            for (int tj = 0; tj < 5; ++tj)
+#pragma unroll
+                for (int c = 0; c < WS; ++c) acc[r][c] = __ffma2_rn(w[tj], v[c + tj], acc[r][c]);
+        }
     }
 }
 
@@ -85,7 +90,7 @@ __device__ __forceinline__ void lce_block(uint32_t vbase, int y, int x, int H, i
 template <int WS, int BR, bool ONE_PATH>
 __device__ __forceinline__ void lce_store_block(uint32_t vbase, const float* stage_o, uint32_t* outb, int r0,
                                                 int y0, int x0, const Dims& dm, int cp, bool lce,
-                                                const float2* wv, float2 bias2) {
+                                                uint32_t wlane, float2 bias2) {
     float2 acc[BR][WS];
 #pragma unroll
     for (int r = 0; r < BR; ++r)
@@ -94,8 +99,8 @@ __device__ __forceinline__ void lce_store_block(uint32_t vbase, const float* sta
     const int y = y0 + r0, x = x0;
     if (lce) {
         const bool inside = y >= 2 && y + BR + 1 < dm.H && x >= 2 && x + WS + 1 < dm.W;
-        if (!ONE_PATH && inside) lce_block<WS, BR, false>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wv, acc);
-        else        lce_block<WS, BR, true>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wv, acc);
+        if (!ONE_PATH && inside) lce_block<WS, BR, false>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wlane, acc);
+        else        lce_block<WS, BR, true>(vbase, y, x, dm.H, dm.W, cp >> 2, (cp & 3) * 4, wlane, acc);
     }
 #pragma unroll
     for (int r = 0; r < BR; ++r)
@@ -120,6 +125,8 @@ __device__ __forceinline__ void img_lce_store(uint32_t vbase, uint32_t wtab, con
                                               int lane, float2 bias2) {
     const int cp = lane & 15;
     const bool lce = wtab != 0u;
+    if (SHAPE == 44) { lce_store_block<4, 2, ONE_PATH>(vbase, stage_o, outb, 2 * (lane >> 4), y0, x0, dm, cp, lce, wtab + cp * 8, bias2); return; }
+    if (SHAPE == 22) { lce_store_block<2, 1, ONE_PATH>(vbase, stage_o, outb, lane >> 4, y0, x0, dm, cp, lce, wtab + cp * 8, bias2); return; }
     float2 wv[25];
     if (lce) {
 #pragma unroll
@@ -128,8 +135,6 @@ __device__ __forceinline__ void img_lce_store(uint32_t vbase, uint32_t wtab, con
     const uint32_t vcol = (cp & 3) * 4;
     const int cq = cp >> 2;
     const int run = (dm.ws & 1) ? 1 : 2;
-    if (SHAPE == 44) { lce_store_block<4, 2, ONE_PATH>(vbase, stage_o, outb, 2 * (lane >> 4), y0, x0, dm, cp, lce, wv, bias2); return; }
-    if (SHAPE == 22) { lce_store_block<2, 1, ONE_PATH>(vbase, stage_o, outb, lane >> 4, y0, x0, dm, cp, lce, wv, bias2); return; }
     const int nruns = rows / run;                             // tiles start at multiples of 16, n_r is a multiple of run
     for (int u2 = lane >> 4; u2 < nruns; u2 += 2) {
         const int t = t0 + u2 * run;
