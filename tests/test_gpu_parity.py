@@ -505,3 +505,48 @@ def test_backward_edge_cases(bra):
     cfg = BraConfig("bwd-dup", 1, 8, 8, 32, 1, 2, 3, "f32")
     idx = np.array([[[[0, 0, 3], [1, 2, 1], [3, 3, 3], [2, 0, 1]]]], dtype=np.int32)
     run_backward_case(bra, cfg, seed=12, index=idx)
+
+
+# ------------------------------------------------------------------ random shapes
+@pytest.mark.parametrize("seed", [11, 12])
+def test_random_shapes_forward_and_backward(bra, seed):
+    """Seeded random problems (head dim 32, bf16): region shapes from 1 x 1 to 8 x 8 and 16-wide, any S in
+    {1, 2, 3, 4, 7}, 1-4 heads, k up to 12, every kernel family that accepts the shape, per-head and
+    shared routing.  Forward against the oracle on the GPU's own index, then every gradient."""
+    rng = np.random.default_rng(seed)
+    ran = 0
+    for it in range(16):
+        S = int(rng.choice([1, 2, 3, 4, 7]))
+        hs, ws = int(rng.integers(1, 9)), int(rng.integers(1, 9))
+        if rng.random() < 0.3:
+            ws, hs = 16, 8 * int(rng.integers(1, 3))
+        heads = int(rng.choice([1, 2, 3, 4]))
+        B = int(rng.choice([1, 2, 3, 40]))
+        if B == 40 and S * S * hs * ws > 300:
+            B = 3
+        k = int(rng.integers(1, min(S * S, 12) + 1))
+        cfg = BraConfig(f"rnd{seed}-{it}", B, S * hs, S * ws, 32 * heads, heads, S, k, "bf16")
+        impl = str(rng.choice(["auto", "img", "mma", "tc"]))
+        shared = bool(rng.random() < 0.2)
+        x = synthetic.make_inputs(cfg, seed=100 * seed + it, with_do=True)
+        t = to_dev(x, cfg)
+        p = problem_of(bra, cfg, impl=IMPLS[impl], shared_routing=shared)
+        ws_buf = bra.workspace(p)
+        try:
+            O, idx, lse = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws_buf)
+        except bra.BraError as e:
+            assert e.code == 7 and impl != "auto"        # that kernel family does not take the shape
+            continue
+        assert bra.bra_device_status(ws_buf) == 0
+        idn = idx.cpu().numpy()
+        O_ref, lse_ref = orc.bra_attend(x["Q"], x["K"], x["V"], idn, x["w"], cfg.heads, cfg.S)
+        check_O(f64(O), O_ref, cfg.dtype)
+        np.testing.assert_allclose(f64(lse), lse_ref, rtol=0, atol=2e-3)
+        g = bra.bra_backward(p, t["Q"], t["K"], t["V"], idx, t["w"], lse, t["dO"], ws=ws_buf, want_bias_grad=True)
+        assert bra.bra_device_status(ws_buf) == 0
+        ref = orc.bra_backward(x["Q"], x["K"], x["V"], idn, x["w"], x["dO"], cfg.heads, cfg.S)
+        for name, a, r in zip(("dQ", "dK", "dV", "d_lce_w", "d_lce_b"), g, ref):
+            scale = max(1.0, np.abs(r).max()) if name.startswith("d_lce") else 1.0
+            assert np.abs(f64(a) - r).max() <= GRAD_MAX * scale, f"{cfg} {impl} {name}"
+        ran += 1
+    assert ran >= 8
