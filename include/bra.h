@@ -14,7 +14,8 @@
  * Common rules for every entry point
  *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte
  *     aligned, dense and contiguous.  The library allocates no device memory
- *     and keeps no state between calls besides cached TMA descriptors.
+ *     and keeps no state between calls besides kernel attributes and launch
+ *     choices remembered per device and problem shape.
  *   - Q, K, V, O, dO, dQ, dK, dV: [B, H, W, C], element type p->dtype, channel
  *     c = head * (C / heads) + j (concat order of Eq. 2).
  *   - Regions: S x S non-overlapping blocks of (H/S) x (W/S) tokens, numbered
