@@ -279,6 +279,45 @@ route_rows_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict_
         sc[j * ROUTE_T_ROWS] = ordered_bits(acc);   // never 0 (NaN is canonical after the + 0): 0 marks "taken"
     }
     int32_t* out = index + (((size_t)b * dm.heads_i + h) * dm.R + i) * dm.topk;
+    if (dm.R <= 64) {
+        // Two levels: the best of each group of eight candidates stays in registers; a rank costs a
+        // maximum over the eight group bests and a rescan of the winner's group only.  Strict
+        // comparisons in ascending order: the first of equal scores wins at both levels.
+        uint32_t gbest[8];
+        int garg[8];
+#pragma unroll
+        for (int gq = 0; gq < 8; ++gq) {
+            gbest[gq] = 0u; garg[gq] = 8 * gq;
+#pragma unroll
+            for (int tq = 0; tq < 8; ++tq) {
+                const int j = 8 * gq + tq;
+                const uint32_t v = j < dm.R ? sc[j * ROUTE_T_ROWS] : 0u;
+                if (v > gbest[gq]) { gbest[gq] = v; garg[gq] = j; }
+            }
+        }
+        for (int m = 0; m < dm.topk; ++m) {
+            uint32_t best = gbest[0];
+            int arg = garg[0];
+#pragma unroll
+            for (int gq = 1; gq < 8; ++gq)
+                if (gbest[gq] > best) { best = gbest[gq]; arg = garg[gq]; }
+            out[m] = arg;
+            sc[arg * ROUTE_T_ROWS] = 0u;
+            const int wg = arg >> 3;
+            uint32_t nb = 0u;
+            int na = 8 * wg;
+#pragma unroll
+            for (int tq = 0; tq < 8; ++tq) {
+                const int j = 8 * wg + tq;
+                const uint32_t v = j < dm.R ? sc[j * ROUTE_T_ROWS] : 0u;
+                if (v > nb) { nb = v; na = j; }
+            }
+#pragma unroll
+            for (int gq = 0; gq < 8; ++gq)
+                if (gq == wg) { gbest[gq] = nb; garg[gq] = na; }
+        }
+        return;
+    }
     for (int m = 0; m < dm.topk; ++m) {
         uint32_t best = 0u;
         int arg = 0;
