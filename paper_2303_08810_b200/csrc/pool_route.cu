@@ -354,6 +354,103 @@ static cudaError_t launch_route_e(const Dims& d, const float* q_mean, const floa
     return e;
 }
 
+// The same routing with half a warp per affinity row (small R, small k): twice the rows per warp,
+// the same instructions per warp.  Lane l of the half scores candidates l, l + 16, ...; the rank
+// rounds reduce over the half's 16 lanes (redux with a half-warp mask).
+constexpr int HALF_ROWS_PER_CTA = 16;
+
+template <int E2>   // score slots per lane: handles R <= 16 * E2
+__global__ void __launch_bounds__(256)
+route_half_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ index, Dims dm) {
+    extern __shared__ float4 kh4[];             // [R][dc + 4] floats, then this CTA's 16 rows of Q^r
+    float* ks = reinterpret_cast<float*>(kh4);
+    pdl_launch_dependents();
+    pdl_wait();                                  // the means come from the kernel before
+    const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
+    const int dc = dm.heads_i == 1 ? dm.C : dm.d;
+    const int c0 = dm.heads_i == 1 ? 0 : h * dm.d;
+    const int ld = dc + 4;
+    const int dc4 = dc >> 2;
+    const float* kb = k_mean + (size_t)b * dm.R * dm.C + c0;
+    // coherent loads: the means come from the pooling kernel this one may overlap
+    for (int i = threadIdx.x; i < dm.R * dc4; i += blockDim.x) {
+        const int r = i / dc4, c4 = i - r * dc4;
+        *reinterpret_cast<float4*>(&ks[r * ld + 4 * c4]) = __ldcg(reinterpret_cast<const float4*>(kb + (size_t)r * dm.C) + c4);
+    }
+    float* qs = ks + (size_t)dm.R * ld;
+    const int row0 = blockIdx.y * HALF_ROWS_PER_CTA;
+    const float* qb = q_mean + ((size_t)b * dm.R + row0) * dm.C + c0;
+    for (int i = threadIdx.x; i < HALF_ROWS_PER_CTA * dc4; i += blockDim.x) {
+        const int r = i / dc4, c4 = i - r * dc4;
+        if (row0 + r < dm.R)
+            *reinterpret_cast<float4*>(&qs[r * dc + 4 * c4]) = __ldcg(reinterpret_cast<const float4*>(qb + (size_t)r * dm.C) + c4);
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, l16 = lane & 15, half = lane >> 4;
+    const int lrow = (threadIdx.x >> 5) * 2 + half;          // this half-warp's row of the CTA
+    const int i = row0 + lrow;
+    const bool live = i < dm.R;                               // both halves run the reductions below; a dead one writes nothing
+    const unsigned hmask = 0xffffu << (16 * half);
+    const float4* qrow = reinterpret_cast<const float4*>(qs + (live ? lrow : 0) * dc);
+    float acc[E2];
+#pragma unroll
+    for (int e = 0; e < E2; ++e) acc[e] = 0.f;
+    for (int c4 = 0; c4 < dc4; ++c4) {
+        const float4 q4 = qrow[c4];
+#pragma unroll
+        for (int e = 0; e < E2; ++e) {
+            const int j = l16 + 16 * e;
+            if (j < dm.R) {
+                const float4 k4 = *reinterpret_cast<const float4*>(&ks[j * ld + 4 * c4]);
+                acc[e] = fmaf(q4.x, k4.x, acc[e]);
+                acc[e] = fmaf(q4.y, k4.y, acc[e]);
+                acc[e] = fmaf(q4.z, k4.z, acc[e]);
+                acc[e] = fmaf(q4.w, k4.w, acc[e]);
+            }
+        }
+    }
+    unsigned long long key[E2];
+#pragma unroll
+    for (int e = 0; e < E2; ++e) {
+        const int j = l16 + 16 * e;
+        key[e] = j < dm.R ? ((unsigned long long)ordered_bits(acc[e]) << 32) | (0xffffffffu - (uint32_t)j) : 0ull;
+    }
+    int32_t* out = index + (((size_t)b * dm.heads_i + h) * dm.R + (live ? i : 0)) * dm.topk;
+    for (int m = 0; m < dm.topk; ++m) {
+        unsigned long long best = key[0];
+#pragma unroll
+        for (int e = 1; e < E2; ++e) best = key[e] > best ? key[e] : best;
+        const uint32_t hi = (uint32_t)(best >> 32);
+        const uint32_t top_hi = __reduce_max_sync(hmask, hi);
+        const uint32_t lo = hi == top_hi ? (uint32_t)best : 0u;
+        const uint32_t top_lo = __reduce_max_sync(hmask, lo);
+        const unsigned long long top = ((unsigned long long)top_hi << 32) | top_lo;
+#pragma unroll
+        for (int e = 0; e < E2; ++e)
+            if (key[e] == top) key[e] = 0ull;            // keys are distinct: they carry the region number
+        if (l16 == 0 && live) out[m] = (int32_t)(0xffffffffu - top_lo);
+    }
+}
+
+static size_t route_half_smem(const Dims& d) {
+    const int dc = d.heads_i == 1 ? d.C : d.d;
+    return sizeof(float) * ((size_t)d.R * (dc + 4) + (size_t)HALF_ROWS_PER_CTA * dc);
+}
+
+template <int E2>
+static cudaError_t launch_route_half(const Dims& d, const float* q_mean, const float* k_mean,
+                                     int32_t* index, cudaStream_t st) {
+    const size_t smem = route_half_smem(d);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(route_half_kernel<E2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    cudaError_t e = launch_kernel(route_half_kernel<E2>, dim3(d.B * d.heads_i, (d.R + HALF_ROWS_PER_CTA - 1) / HALF_ROWS_PER_CTA),
+                                  dim3(256), smem, st, /*after_own_kernel=*/true, q_mean, k_mean, index, d);
+    count_launch();
+    return e;
+}
+
 static size_t route_rows_smem(const Dims& d) {
     const int dc = d.heads_i == 1 ? d.C : d.d;
     return sizeof(float) * (size_t)d.R * (dc + 4) + sizeof(uint32_t) * (size_t)d.R * ROUTE_T_ROWS;
@@ -382,6 +479,10 @@ cudaError_t launch_route(const Dims& d, const float* q_mean, const float* k_mean
         return dc == 32 ? launch_route_rows<8>(d, q_mean, k_mean, index, st)
                         : launch_route_rows<0>(d, q_mean, k_mean, index, st);
     }
+    // small R and k: half a warp per row
+    if (d.R <= 64 && d.topk <= 8 && route_half_smem(d) <= 100 * 1024)
+        return d.R <= 32 ? launch_route_half<2>(d, q_mean, k_mean, index, st)
+                         : launch_route_half<4>(d, q_mean, k_mean, index, st);
     if (d.R <= 32) return launch_route_e<1>(d, q_mean, k_mean, index, st);
     if (d.R <= 64) return launch_route_e<2>(d, q_mean, k_mean, index, st);
     if (d.R <= 128) return launch_route_e<4>(d, q_mean, k_mean, index, st);
