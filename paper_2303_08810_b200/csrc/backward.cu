@@ -398,23 +398,32 @@ bwd_dw_partial_staged_kernel(const T* __restrict__ V, const T* __restrict__ dO, 
     }
 }
 
-// Final sum over the partials: 32 outputs per CTA, 8 threads per output each taking every
-// eighth partial in order; the eight slice sums are then added in order.
-__global__ void __launch_bounds__(256)
+// Final sum over the partials: 32 outputs per CTA, 32 threads per output each taking every
+// 32nd partial in order (four loads in flight); the slice sums are then added in order.
+constexpr int DW_SLICES = 32;
+__global__ void __launch_bounds__(32 * DW_SLICES)
 bwd_dw_final_kernel(const float* __restrict__ part, int blocks,
                     float* __restrict__ d_lce_w, float* __restrict__ d_lce_b, Dims dm) {
-    __shared__ float sl[8][32];
+    __shared__ float sl[DW_SLICES][32];
     const int o = blockIdx.x * 32 + threadIdx.x;   // (channel, slot)
     const int slice = threadIdx.y;
+    const size_t stride = (size_t)dm.C * 26;
     float s = 0.f;
-    if (o < dm.C * 26)
-        for (int p = slice; p < blocks; p += 8) s += part[(size_t)p * dm.C * 26 + o];
+    if (o < dm.C * 26) {
+        int p = slice;
+        for (; p + 3 * DW_SLICES < blocks; p += 4 * DW_SLICES) {
+            const float a0 = part[(size_t)p * stride + o], a1 = part[(size_t)(p + DW_SLICES) * stride + o];
+            const float a2 = part[(size_t)(p + 2 * DW_SLICES) * stride + o], a3 = part[(size_t)(p + 3 * DW_SLICES) * stride + o];
+            s += a0; s += a1; s += a2; s += a3;
+        }
+        for (; p < blocks; p += DW_SLICES) s += part[(size_t)p * stride + o];
+    }
     sl[slice][threadIdx.x] = s;
     __syncthreads();
     if (slice == 0 && o < dm.C * 26) {
         float t = sl[0][threadIdx.x];
 #pragma unroll
-        for (int q = 1; q < 8; ++q) t += sl[q][threadIdx.x];
+        for (int q = 1; q < DW_SLICES; ++q) t += sl[q][threadIdx.x];
         const int c = o / 26, k = o % 26;
         if (k < 25) { if (d_lce_w) d_lce_w[c * 25 + k] = t; }
         else if (d_lce_b) d_lce_b[c] = t;
@@ -496,7 +505,7 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
         }
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        bwd_dw_final_kernel<<<(d.C * 26 + 31) / 32, dim3(32, 8), 0, st>>>(part, nblk, d.lce ? d_lce_w : nullptr, d_lce_b, d);
+        bwd_dw_final_kernel<<<(d.C * 26 + 31) / 32, dim3(32, DW_SLICES), 0, st>>>(part, nblk, d.lce ? d_lce_w : nullptr, d_lce_b, d);
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
