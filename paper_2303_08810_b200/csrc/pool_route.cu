@@ -64,6 +64,48 @@ pool_kernel(const T* __restrict__ Q, const T* __restrict__ K,
     }
 }
 
+// Regions eight token rows high: two threads per (column, 16-byte vector), four rows each, so that a
+// region is summed by twice the threads with half the work each (short CTAs turn over faster, which
+// is what this latency-bound scan needs).  Row halves are added lower half first.
+template <typename T>
+__global__ void __launch_bounds__(256)
+pool_split_kernel(const T* __restrict__ Q, const T* __restrict__ K,
+                  float* __restrict__ q_mean, float* __restrict__ k_mean, Dims dm) {
+    constexpr int VEC = Vec<T>::n;
+    extern __shared__ float part[];   // [2][ws][C]
+    pdl_launch_dependents();
+    const int r = blockIdx.x, b = blockIdx.y;
+    const int ry = r / dm.S, rx = r - ry * dm.S;
+    const T* src = blockIdx.z == 0 ? Q : K;
+    float* dst = blockIdx.z == 0 ? q_mean : k_mean;
+    const int cvecs = dm.C / VEC;
+    const int items = dm.ws * cvecs;
+    const size_t row_elems = (size_t)dm.W * dm.C;
+    const int wsC = dm.ws * dm.C;
+    const int it = threadIdx.x % items, yh = threadIdx.x / items;        // blockDim.x == 2 * items
+    const T* p = src + ((size_t)b * dm.H + (size_t)ry * dm.hs + 4 * yh) * row_elems + (size_t)rx * dm.ws * dm.C + (size_t)it * VEC;
+    float v[4][VEC];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) load_row<VEC>(p + (size_t)u * row_elems, v[u]);
+    float acc[VEC];
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) acc[i] += v[u][i];
+#pragma unroll
+    for (int i = 0; i < VEC; i += 4)
+        *reinterpret_cast<float4*>(&part[yh * wsC + it * VEC + i]) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+    __syncthreads();
+    const float inv = 1.0f / (float)dm.n_r;
+    for (int c = threadIdx.x; c < dm.C; c += blockDim.x) {
+        float s = 0.f;
+        for (int x = 0; x < dm.ws; ++x) s += part[x * dm.C + c] + part[wsC + x * dm.C + c];
+        dst[((size_t)b * dm.R + r) * dm.C + c] = s * inv;
+    }
+}
+
 cudaError_t launch_pool(const Dims& d, int dtype, const void* Q, const void* K,
                         float* q_mean, float* k_mean, cudaStream_t st) {
     const int vec = dtype == BRA_BF16 ? 8 : 4;
@@ -72,6 +114,16 @@ cudaError_t launch_pool(const Dims& d, int dtype, const void* Q, const void* K,
     size_t smem = sizeof(float) * (size_t)d.ws * d.C;
     dim3 grid(d.R, d.B, 2);
     cudaError_t e;
+    if (d.hs == 8 && 2 * items <= 256 && 2 * smem <= 48 * 1024) {
+        if (dtype == BRA_BF16)
+            pool_split_kernel<__nv_bfloat16><<<grid, 2 * items, 2 * smem, st>>>(
+                static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K), q_mean, k_mean, d);
+        else
+            pool_split_kernel<float><<<grid, 2 * items, 2 * smem, st>>>(
+                static_cast<const float*>(Q), static_cast<const float*>(K), q_mean, k_mean, d);
+        count_launch();
+        return cudaGetLastError();
+    }
     if (dtype == BRA_BF16) {
         if (smem > 48 * 1024 &&
             (e = cudaFuncSetAttribute(pool_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
