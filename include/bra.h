@@ -25,8 +25,11 @@
  *     p->shared_routing != 0).  Row i lists the key regions that the queries of
  *     region i attend to.  It is a list: any order, duplicates count twice.
  *   - ws: scratch of at least bra_workspace_bytes(p) bytes, 256-byte aligned.
- *     Its first bytes hold a device status word; calls that share a ws must
- *     be ordered on one stream.
+ *     It holds a device status block and, for the one-launch forward, job
+ *     counters and per-image flags that the kernels expect to find ZERO and
+ *     leave zero: before its first use fill ws with zeros or call
+ *     bra_workspace_init().  bra_device_status() restores that state when it
+ *     reports an error.  Calls that share a ws must be ordered on one stream.
  *   - Every call is asynchronous on `stream` (a cudaStream_t passed as void*).
  *   - Errors a host check can find return synchronously, nothing launched,
  *     outputs untouched.  Errors only the device can see (an out-of-range
@@ -71,6 +74,15 @@ typedef enum bra_impl {
                            shared memory (C/heads == 32, H*W <= ~1500 tokens): small maps, small regions */
 } bra_impl;
 
+/*
+ * Failure injection for tests of the error path (no GPU fault, trap or hang is involved).
+ * BRA_INJECT_HOLD_ROUTE_FLAGS: in the one-launch forward (bra_forward on 8 x 8-token regions with
+ * topk = 1) the routing step keeps the per-image "routed" flags down, so every attention job's bounded
+ * wait on them runs out after a few thousand polls with no tensor-core work in flight; the kernel returns
+ * normally, O is not written and bra_device_status() reports BRA_ERR_TIMEOUT.  Ignored by every other path.
+ */
+typedef enum bra_inject { BRA_INJECT_NONE = 0, BRA_INJECT_HOLD_ROUTE_FLAGS = 1 } bra_inject;
+
 /* Problem statement in the notation of Algorithm 1 (H, W, C, S, k) plus batch and heads. */
 typedef struct bra_problem {
     int32_t B, H, W, C;     /* batch, feature-map height and width, channels */
@@ -83,10 +95,19 @@ typedef struct bra_problem {
                                1: one index for all heads (Eq. 4 read over all C channels) */
     int32_t lce_ksize;      /* 5: add LCE(V) (Eq. 7); 0: attention term only */
     int32_t impl;           /* bra_impl */
+    int32_t inject;         /* bra_inject: 0 in production */
 } bra_problem;
 
 /* Scratch size in bytes every call on problem p needs (0 if p is invalid). Host only. */
 size_t bra_workspace_bytes(const bra_problem* p);
+
+/*
+ * Puts ws into the state the kernels expect: status block, job counters and per-image flags zero
+ * (asynchronous memsets on `stream`; the rest of ws needs no initial value).  Needed once before the
+ * first use of a ws that was not zero-filled.  (Housekeeping of this library: Algorithm 1 has no
+ * counterpart.)
+ */
+bra_status bra_workspace_init(const bra_problem* p, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Region-to-region routing (Section 3.2: per-region average; Eq. 4; Eq. 5).
@@ -151,7 +172,10 @@ bra_status bra_attend(const bra_problem* p, const void* Q, const void* K, const 
                       void* O, float* lse, void* ws, size_t ws_bytes, void* stream);
 
 /*
- * Algorithm 1 from the projected Q, K, V on: bra_route then bra_attend in one call.
+ * Algorithm 1 from the projected Q, K, V on: bra_route then bra_attend in one call; same results,
+ * bit for bit, as the two calls.  For bf16 problems with head dim 32, 8 x 8-token regions, topk = 1,
+ * per-head routing, at most 64 regions and C <= 128 the whole call is ONE kernel launch (pooling,
+ * Eq. 4, Eq. 5 and the attention overlap inside it); other problems chain the library's kernels.
  *   index    out  may be NULL (then kept in ws only)
  *   lse      out  may be NULL
  */
@@ -181,7 +205,9 @@ bra_status bra_backward(const bra_problem* p, const void* Q, const void* K, cons
 /*
  * Synchronises `stream`, then returns and clears the first device-detected
  * error recorded in ws (BRA_OK, BRA_ERR_INDEX, BRA_ERR_TIMEOUT, or BRA_ERR_CUDA
- * if the synchronisation itself failed).  ws must have been used by an earlier call.
+ * if the synchronisation itself failed).  When it reports an error it also puts the
+ * counters and flags in ws back to zero (as bra_workspace_init does), so the next call
+ * starts clean.  ws must have been initialised and used by an earlier call.
  */
 bra_status bra_device_status(void* ws, void* stream);
 

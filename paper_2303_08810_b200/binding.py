@@ -25,6 +25,7 @@ class BraProblem(ctypes.Structure):
         ("B", c_int32), ("H", c_int32), ("W", c_int32), ("C", c_int32),
         ("heads", c_int32), ("S", c_int32), ("topk", c_int32), ("dtype", c_int32),
         ("scale", c_float), ("shared_routing", c_int32), ("lce_ksize", c_int32), ("impl", c_int32),
+        ("inject", c_int32),
     ]
 
     @property
@@ -43,7 +44,8 @@ class BraError(RuntimeError):
 
 
 def library_path() -> str:
-    return os.path.join(os.path.dirname(os.path.abspath(__file__)), _LIB_NAME)
+    """The built library next to this file, or the file BRA_LIBRARY_PATH names (to try another build)."""
+    return os.environ.get("BRA_LIBRARY_PATH") or os.path.join(os.path.dirname(os.path.abspath(__file__)), _LIB_NAME)
 
 
 def load_library():
@@ -61,6 +63,8 @@ def load_library():
     v = c_void_p
     lib.bra_workspace_bytes.restype = c_size_t
     lib.bra_workspace_bytes.argtypes = [P]
+    lib.bra_workspace_init.restype = c_int32
+    lib.bra_workspace_init.argtypes = [P, v, c_size_t, v]
     lib.bra_route.restype = c_int32
     lib.bra_route.argtypes = [P, v, v, v, v, v, v, c_size_t, v]
     lib.bra_route_static.restype = c_int32
@@ -96,10 +100,10 @@ def last_launch_count() -> int:
 
 
 def make_problem(B, H, W, C, heads, S, topk, dtype="bf16", scale=0.0, shared_routing=False,
-                 lce=True, impl=IMPL_AUTO) -> BraProblem:
+                 lce=True, impl=IMPL_AUTO, inject=0) -> BraProblem:
     dt = {"f32": F32, "bf16": BF16, F32: F32, BF16: BF16}[dtype]
     return BraProblem(B, H, W, C, heads, S, topk, dt, float(scale), int(bool(shared_routing)),
-                      5 if lce else 0, int(impl))
+                      5 if lce else 0, int(impl), int(inject))
 
 
 def workspace_bytes(p: BraProblem) -> int:
@@ -120,6 +124,13 @@ def workspace(p: BraProblem, device="cuda"):
     if n == 0:
         raise BraError(2, "bra_workspace_bytes")
     return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def workspace_init(p: BraProblem, ws, stream=None):
+    """bra_workspace_init: status block, job counters and flags of `ws` set to zero."""
+    _check(load_library().bra_workspace_init(ctypes.byref(p), _ptr(ws), ws.numel(), _stream(stream)),
+           "bra_workspace_init")
+    return ws
 
 
 def _ptr(t):

@@ -327,16 +327,21 @@ static cudaError_t img_occupancy(AttendImgKernel kernel, int nw, int smem_bytes,
 
 cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
                               const int32_t* index, const float* lce_w, const float* lce_b,
-                              void* O, float* lse, int32_t* status, cudaStream_t st) {
+                              void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel) {
     // Warps per CTA and register variant (SMALL: up to ~200 registers, CTAs of at most 5 warps): among
     // the choices that let every CTA of the grid be resident at once, the one with the most warps per
     // SM (the roomier variant on a tie); if none does, the most warps per SM.  Remembered per shape.
     const long long grid = (long long)d.B * d.heads;
     const int shape = img_region_shape(d);
-    static thread_local struct { long long grid; int N, ents, nw; bool small; } memo = {0, 0, 0, 0, false};
+    // the choice depends on the whole problem shape (kernel instantiation, shared-memory size) and on the device
+    struct Memo { long long grid; int dev, H, W, C, S, topk, lce, nw; bool small; };
+    static thread_local Memo memo = {0, -1, 0, 0, 0, 0, 0, 0, 0, false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     int best_nw = 0;
     bool best_small = false;
-    if (memo.nw && memo.grid == grid && memo.N == d.N && memo.ents == d.R * d.topk) {
+    if (memo.nw && memo.grid == grid && memo.dev == dev && memo.H == d.H && memo.W == d.W && memo.C == d.C &&
+        memo.S == d.S && memo.topk == d.topk && memo.lce == d.lce) {
         best_nw = memo.nw;
         best_small = memo.small;
     } else {
@@ -359,13 +364,13 @@ cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const
             }
         }
         if (!best_nw) return cudaErrorInvalidConfiguration;
-        memo.grid = grid; memo.N = d.N; memo.ents = d.R * d.topk; memo.nw = best_nw; memo.small = best_small;
+        memo = Memo{grid, dev, d.H, d.W, d.C, d.S, d.topk, d.lce, best_nw, best_small};
     }
     const ImgGeom g = img_geom(d, best_nw);
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(Q);
     const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(K);
     const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(V);
-    const bool pdl = take_after_own_kernel();
+    const bool pdl = after_own_kernel;
     AttendImgKernel kernel = img_kernel(best_small, shape);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
     if (e != cudaSuccess) return e;

@@ -316,16 +316,18 @@ bool attend_mma_supported(const Dims& d, int dtype) {
 
 cudaError_t launch_attend_mma(const Dims& d, const void* Q, const void* K, const void* V,
                               const int32_t* index, const float* lce_w, const float* lce_b,
-                              void* O, float* lse, int32_t* status, cudaStream_t st) {
+                              void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel) {
     const MmaGeom g = mma_geom(d);
     static PerDeviceMax smem_set;
-    if (g.smem_bytes > 48 * 1024 && smem_set.raise(g.smem_bytes)) {
-        cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
-        if (e != cudaSuccess) return e;
-    }
+    cudaError_t e = cudaSuccess;
+    if (g.smem_bytes > 48 * 1024)
+        e = smem_set.ensure(g.smem_bytes, [&] {
+            return cudaFuncSetAttribute(attend_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
+        });
+    if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)((long long)d.B * d.R * d.heads * g.chunks);
-    cudaError_t e = launch_kernel(attend_mma_kernel, dim3(grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st,
-                                  take_after_own_kernel(),
+    e = launch_kernel(attend_mma_kernel, dim3(grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st,
+                                  after_own_kernel,
                                   static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
                                   static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b,
                                   static_cast<__nv_bfloat16*>(O), lse, status, d, g);

@@ -337,22 +337,22 @@ bool attend_tc_wide_supported(const Dims& d, int dtype) {
 
 cudaError_t launch_attend_tc_wide(const Dims& d, const void* Q, const void* K, const void* V,
                                   const int32_t* index, const float* lce_w, const float* lce_b,
-                                  void* O, float* lse, int32_t* status, cudaStream_t st) {
-    static PerDeviceMax attr_set;
-    if (attr_set.raise(1)) {
-        cudaError_t e = cudaFuncSetAttribute(attend_tc_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tw::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(attend_tc_wide_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-    }
+                                  void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel) {
+    static PerDeviceOnce attr_set;
+    cudaError_t e = attr_set.run([] {
+        cudaError_t a = cudaFuncSetAttribute(attend_tc_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tw::SMEM_BYTES);
+        if (a != cudaSuccess) return a;
+        return cudaFuncSetAttribute(attend_tc_wide_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    });
+    if (e != cudaSuccess) return e;
     int dev = 0, sms = 1;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
     const int tiles = d.B * d.R * d.heads * (d.hs / tw::RT);
     const int resident = sms * 4;
     const unsigned grid = (unsigned)(tiles < resident ? tiles : resident);
-    cudaError_t e = launch_kernel(attend_tc_wide_kernel, dim3(grid), dim3(tw::THREADS), tw::SMEM_BYTES, st,
-                                  take_after_own_kernel(),
+    e = launch_kernel(attend_tc_wide_kernel, dim3(grid), dim3(tw::THREADS), tw::SMEM_BYTES, st,
+                                  after_own_kernel,
                                   static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
                                   static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b,
                                   static_cast<__nv_bfloat16*>(O), lse, status, d, tiles);

@@ -430,15 +430,12 @@ bwd_dw_final_kernel(const float* __restrict__ part, int blocks,
     }
 }
 
-static thread_local int g_bwd_impl = BRA_IMPL_AUTO;
-void hint_backward_impl(int impl) { g_bwd_impl = impl; }
-
 bool backward_supported(const Dims& d) {
     return (d.d == 16 || d.d == 32 || d.d == 64) && d.R <= 1000;
 }
 
 template <typename T, int D>
-static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, const void* V,
+static cudaError_t launch_bwd_t(const Dims& d, int impl, const void* Q, const void* K, const void* V,
                                 const int32_t* index, const float* lce_w, const float* lse,
                                 const void* dO, void* dQ, void* dK, void* dV,
                                 float* d_lce_w, float* d_lce_b, char* ws, const WsLayout& L,
@@ -455,8 +452,8 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
     // bf16, head dim 32: tensor-core kernels.  Small maps with enough (image, head) pairs to fill the
     // GPU keep a whole slice resident; the rest stream blocks through shared memory.
     const bool img_ok = sizeof(T) == 2 && backward_img_supported(d, BRA_BF16);
-    const bool use_img = img_ok && (g_bwd_impl == BRA_IMPL_IMG ||
-                                    (g_bwd_impl == BRA_IMPL_AUTO && (long long)d.B * d.heads >= 64));
+    const bool use_img = img_ok && (impl == BRA_IMPL_IMG ||
+                                    (impl == BRA_IMPL_AUTO && (long long)d.B * d.heads >= 64));
     if (!use_img) {
         const int thr = 256;
         const size_t idx_bytes = sizeof(int32_t) * (size_t)d.R * d.topk;
@@ -470,7 +467,7 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
         // the dQ kernel of this family also writes the inverse routing index
         if ((e = launch_backward_img(d, Q, K, V, index, inv_off, inv_list, lce_w, lse, dO, dQ, dK, dV,
                                      delta, status, st)) != cudaSuccess) return e;
-    } else if (sizeof(T) == 2 && g_bwd_impl != BRA_IMPL_SIMT && backward_mma_supported(d, BRA_BF16)) {
+    } else if (sizeof(T) == 2 && impl != BRA_IMPL_SIMT && backward_mma_supported(d, BRA_BF16)) {
         // head dim 32, bf16: the two tensor-core kernels (dQ + delta, then dK / dV)
         if ((e = launch_backward_mma(d, Q, K, V, index, inv_off, inv_list, lce_w, lse, dO, dQ, dK, dV,
                                      delta, status, st)) != cudaSuccess) return e;
@@ -495,10 +492,12 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
         const size_t dw_smem = (size_t)(2 * rpb + 4) * d.W * d.C * sizeof(T);
         if (dw_smem <= 100 * 1024 && ((size_t)d.W * d.C * sizeof(T)) % 16 == 0) {
             static PerDeviceMax dw_set;
-            if (dw_smem > 48 * 1024 && dw_set.raise((int)dw_smem)) {
-                if ((e = cudaFuncSetAttribute(bwd_dw_partial_staged_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)dw_smem)) != cudaSuccess) return e;
-            }
+            if (dw_smem > 48 * 1024 &&
+                (e = dw_set.ensure((int)dw_smem, [&] {
+                     return cudaFuncSetAttribute(bwd_dw_partial_staged_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)dw_smem);
+                 })) != cudaSuccess)
+                return e;
             bwd_dw_partial_staged_kernel<T><<<nblk, dim3(cpx, DW_TI), dw_smem, st>>>(v, go, part, rpb, d);
         } else {
             bwd_dw_partial_kernel<T><<<nblk, dim3(cpx, DW_TI), 0, st>>>(v, go, part, rpb, d);
@@ -513,27 +512,27 @@ static cudaError_t launch_bwd_t(const Dims& d, const void* Q, const void* K, con
 }
 
 template <typename T>
-static cudaError_t launch_bwd_d(const Dims& d, const void* Q, const void* K, const void* V,
+static cudaError_t launch_bwd_d(const Dims& d, int impl, const void* Q, const void* K, const void* V,
                                 const int32_t* index, const float* lce_w, const float* lse,
                                 const void* dO, void* dQ, void* dK, void* dV,
                                 float* d_lce_w, float* d_lce_b, char* ws, const WsLayout& L,
                                 cudaStream_t st) {
     switch (d.d) {
-        case 16: return launch_bwd_t<T, 16>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
-        case 32: return launch_bwd_t<T, 32>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
-        case 64: return launch_bwd_t<T, 64>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+        case 16: return launch_bwd_t<T, 16>(d, impl, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+        case 32: return launch_bwd_t<T, 32>(d, impl, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+        case 64: return launch_bwd_t<T, 64>(d, impl, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
     }
     return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_backward(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
+cudaError_t launch_backward(const Dims& d, int dtype, int impl, const void* Q, const void* K, const void* V,
                             const int32_t* index, const float* lce_w, const float* lse,
                             const void* dO, void* dQ, void* dK, void* dV,
                             float* d_lce_w, float* d_lce_b,
                             char* ws, const WsLayout& L, cudaStream_t st) {
     if (dtype == BRA_BF16)
-        return launch_bwd_d<__nv_bfloat16>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
-    return launch_bwd_d<float>(d, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+        return launch_bwd_d<__nv_bfloat16>(d, impl, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
+    return launch_bwd_d<float>(d, impl, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV, d_lce_w, d_lce_b, ws, L, st);
 }
 
 }  // namespace bra

@@ -479,12 +479,16 @@ cudaError_t launch_backward_mma(const Dims& d, const void* Q, const void* K, con
     const BwdGeom a = bwd_geom(d, false), b = bwd_geom(d, true);
     static PerDeviceMax smem_a, smem_b;
     cudaError_t e;
-    if (a.smem_bytes > 48 * 1024 && smem_a.raise(a.smem_bytes)) {
-        if ((e = cudaFuncSetAttribute(bwd_dq_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, a.smem_bytes)) != cudaSuccess) return e;
-    }
-    if (b.smem_bytes > 48 * 1024 && smem_b.raise(b.smem_bytes)) {
-        if ((e = cudaFuncSetAttribute(bwd_dkv_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, b.smem_bytes)) != cudaSuccess) return e;
-    }
+    if (a.smem_bytes > 48 * 1024 &&
+        (e = smem_a.ensure(a.smem_bytes, [&] {
+             return cudaFuncSetAttribute(bwd_dq_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, a.smem_bytes);
+         })) != cudaSuccess)
+        return e;
+    if (b.smem_bytes > 48 * 1024 &&
+        (e = smem_b.ensure(b.smem_bytes, [&] {
+             return cudaFuncSetAttribute(bwd_dkv_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, b.smem_bytes);
+         })) != cudaSuccess)
+        return e;
     const unsigned grid = (unsigned)((long long)d.B * d.R * d.heads * a.g.chunks);
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(Q);
     const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(K);

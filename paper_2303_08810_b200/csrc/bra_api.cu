@@ -25,6 +25,7 @@ WsLayout ws_layout(const Dims& d) {
     while (blocks > 1024 && blocks % 2 == 0) blocks /= 2;
     L.dw_blocks = blocks;
     L.dw_part = off;  off += align256(sizeof(float) * (size_t)blocks * d.C * 26);
+    L.sync = off;     off += align256(sizeof(int32_t) * 2 * (size_t)d.B);
     L.total = off;
     return L;
 }
@@ -40,6 +41,7 @@ static bra_status make_dims(const bra_problem* p, Dims* out) {
     if (p->dtype != BRA_F32 && p->dtype != BRA_BF16) return BRA_ERR_DTYPE;
     if (p->lce_ksize != 0 && p->lce_ksize != 5) return BRA_ERR_UNSUPPORTED;
     if (p->impl < BRA_IMPL_AUTO || p->impl > BRA_IMPL_IMG) return BRA_ERR_UNSUPPORTED;
+    if (p->inject != BRA_INJECT_NONE && p->inject != BRA_INJECT_HOLD_ROUTE_FLAGS) return BRA_ERR_UNSUPPORTED;
     Dims d;
     d.B = p->B; d.H = p->H; d.W = p->W; d.C = p->C; d.heads = p->heads; d.S = p->S; d.topk = p->topk;
     d.d = p->C / p->heads;
@@ -60,9 +62,6 @@ static bra_status make_dims(const bra_problem* p, Dims* out) {
 // For translation units that add entry points of their own.
 bra_status check_problem(const bra_problem* p, Dims* out) { return make_dims(p, out); }
 void reset_launch_count() { g_launches = 0; }
-static thread_local bool g_after_own = false;
-void hint_after_own_kernel(bool yes) { g_after_own = yes; }
-bool take_after_own_kernel() { const bool v = g_after_own; g_after_own = false; return v; }
 
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -104,14 +103,14 @@ static bra_status run_route(const Dims& d, int dtype, const void* Q, const void*
 static bra_status run_attend(Path path, const Dims& d, int dtype, const void* Q, const void* K,
                              const void* V, const int32_t* index, const float* lce_w,
                              const float* lce_b, void* O, float* lse, int32_t* status,
-                             cudaStream_t st) {
+                             cudaStream_t st, bool after_own_kernel) {
     cudaError_t e = cudaErrorInvalidValue;
     switch (path) {
         case PATH_SIMT: e = launch_attend_simt(d, dtype, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
-        case PATH_MMA:  e = launch_attend_mma(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
-        case PATH_TC:   e = launch_attend_tc(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
-        case PATH_TC_WIDE: e = launch_attend_tc_wide(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
-        case PATH_IMG:  e = launch_attend_img(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st); break;
+        case PATH_MMA:  e = launch_attend_mma(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st, after_own_kernel); break;
+        case PATH_TC:   e = launch_attend_tc(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st, after_own_kernel); break;
+        case PATH_TC_WIDE: e = launch_attend_tc_wide(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st, after_own_kernel); break;
+        case PATH_IMG:  e = launch_attend_img(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st, after_own_kernel); break;
         default: return BRA_ERR_UNSUPPORTED;
     }
     return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;
@@ -166,7 +165,7 @@ bra_status bra_attend(const bra_problem* p, const void* Q, const void* K, const 
     if (path == PATH_NONE) return BRA_ERR_UNSUPPORTED;
     char* w = static_cast<char*>(ws);
     return run_attend(path, d, p->dtype, Q, K, V, index, lce_w, lce_b, O, lse,
-                      reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(stream));
+                      reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(stream), false);
 }
 
 bra_status bra_forward(const bra_problem* p, const void* Q, const void* K, const void* V,
@@ -189,14 +188,19 @@ bra_status bra_forward(const bra_problem* p, const void* Q, const void* K, const
     char* w = static_cast<char*>(ws);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t* idx = index ? index : reinterpret_cast<int32_t*>(w + L.index);
-    s = run_route(d, p->dtype, Q, K, reinterpret_cast<float*>(w + L.q_mean),
-                  reinterpret_cast<float*>(w + L.k_mean), idx, st);
+    int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
+    float* qm = reinterpret_cast<float*>(w + L.q_mean);
+    float* km = reinterpret_cast<float*>(w + L.k_mean);
+    // pooling, routing and attention in one launch where the tcgen05 kernel can do all three
+    static const bool no_fused = getenv("BRA_NO_FUSED") != nullptr;    // debugging aid: the three-launch chain
+    if (path == PATH_TC && !no_fused && forward_tc_supported(d, p->dtype)) {
+        const cudaError_t e = launch_forward_tc(d, Q, K, V, lce_w, lce_b, O, idx, lse, qm, km, status,
+                                                reinterpret_cast<int32_t*>(w + L.sync), p->inject, st);
+        return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;
+    }
+    s = run_route(d, p->dtype, Q, K, qm, km, idx, st);
     if (s != BRA_OK) return s;
-    hint_after_own_kernel(true);
-    s = run_attend(path, d, p->dtype, Q, K, V, idx, lce_w, lce_b, O, lse,
-                   reinterpret_cast<int32_t*>(w + L.status), st);
-    hint_after_own_kernel(false);
-    return s;
+    return run_attend(path, d, p->dtype, Q, K, V, idx, lce_w, lce_b, O, lse, status, st, true);
 }
 
 bra_status bra_backward(const bra_problem* p, const void* Q, const void* K, const void* V,
@@ -217,22 +221,41 @@ bra_status bra_backward(const bra_problem* p, const void* Q, const void* K, cons
     WsLayout L;
     if ((s = check_ws(d, ws, ws_bytes, &L)) != BRA_OK) return s;
     if (!backward_supported(d)) return BRA_ERR_UNSUPPORTED;
-    hint_backward_impl(p->impl);
-    cudaError_t e = launch_backward(d, p->dtype, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV,
+    cudaError_t e = launch_backward(d, p->dtype, p->impl, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV,
                                     d_lce_w, d_lce_b, static_cast<char*>(ws), L,
                                     static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;
 }
 
+bra_status bra_workspace_init(const bra_problem* p, void* ws, size_t ws_bytes, void* stream) {
+    g_launches = 0;
+    Dims d;
+    bra_status s = make_dims(p, &d);
+    if (s != BRA_OK) return s;
+    WsLayout L;
+    if ((s = check_ws(d, ws, ws_bytes, &L)) != BRA_OK) return s;
+    char* w = static_cast<char*>(ws);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the status block and the counters / flags of the one-launch forward; the rest is written before it is read
+    if (cudaMemsetAsync(w + L.status, 0, 256, st) != cudaSuccess) return BRA_ERR_CUDA;
+    if (cudaMemsetAsync(w + L.sync, 0, L.total - L.sync, st) != cudaSuccess) return BRA_ERR_CUDA;
+    return BRA_OK;
+}
+
 bra_status bra_device_status(void* ws, void* stream) {
     if (!ws) return BRA_ERR_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int32_t host[2] = {0, 0};
+    int32_t host[4] = {0, 0, 0, 0};     // code, detail; offset and size of the one-launch forward's counters
     if (cudaMemcpyAsync(host, ws, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return BRA_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return BRA_ERR_CUDA;
     if (host[0] != 0) {
-        if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return BRA_ERR_CUDA;
+        // a kernel that gave up leaves its job counter, per-image counters and flags as they were: clear
+        // them with the error, so that the next call on this ws starts clean
+        if (cudaMemsetAsync(ws, 0, 256, st) != cudaSuccess) return BRA_ERR_CUDA;
+        if (host[2] >= 256 && host[3] > 0 &&
+            cudaMemsetAsync(static_cast<char*>(ws) + host[2], 0, (size_t)host[3], st) != cudaSuccess)
+            return BRA_ERR_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return BRA_ERR_CUDA;
     }
     if (host[0] < 0 || host[0] > BRA_ERR_TIMEOUT) return BRA_ERR_CUDA;
@@ -259,6 +282,6 @@ const char* bra_status_string(bra_status s) {
     return "unknown status";
 }
 
-int32_t bra_version(void) { return 100; }
+int32_t bra_version(void) { return 200; }
 
 }  // extern "C"

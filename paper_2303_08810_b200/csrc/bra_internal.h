@@ -8,6 +8,8 @@
 #include <stddef.h>
 #include <stdlib.h>
 
+#include <mutex>
+
 #include "../../include/bra.h"
 
 namespace bra {
@@ -35,6 +37,7 @@ struct WsLayout {
     size_t inv_off;     // int32 [B,heads_i,R+1] CSR offsets of the inverse routing index
     size_t inv_list;    // int32 [B,heads_i,R*topk] query regions routed to each key region
     size_t dw_part;     // fp32 [dw_blocks, C*26] partial LCE weight / bias gradients
+    size_t sync;        // int32 [2,B] one-launch forward: pooled units per image, "image routed" flags (zero between calls)
     size_t total;
     int dw_blocks;
 };
@@ -44,10 +47,6 @@ WsLayout ws_layout(const Dims& d);
 // Host-side bookkeeping of kernel launches for bra_last_launch_count().
 void count_launch(int n = 1);
 void reset_launch_count();
-// bra_forward tells the attend launcher that the kernel before it in the stream is the
-// library's own routing kernel (so the launch may overlap its tail); read-and-clear.
-void hint_after_own_kernel(bool yes);
-bool take_after_own_kernel();
 
 // Validate a problem statement and fill the derived dimensions.
 bra_status check_problem(const bra_problem* p, Dims* out);
@@ -68,21 +67,30 @@ cudaError_t launch_attend_simt(const Dims& d, int dtype, const void* Q, const vo
 bool attend_mma_supported(const Dims& d, int dtype);
 cudaError_t launch_attend_mma(const Dims& d, const void* Q, const void* K, const void* V,
                               const int32_t* index, const float* lce_w, const float* lce_b,
-                              void* O, float* lse, int32_t* status, cudaStream_t st);
+                              void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel);
 
+// after_own_kernel (here and below): the kernel before this one in the stream is the library's own
+// routing kernel, so the launch may overlap its tail (programmatic dependent launch)
 bool attend_tc_supported(const Dims& d, int dtype);
 cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const void* V,
                              const int32_t* index, const float* lce_w, const float* lce_b,
-                             void* O, float* lse, int32_t* status, cudaStream_t st);
+                             void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel);
+
+// Algorithm 1 in one launch (pooling, routing and attention of 8 x 8-token regions, topk = 1)
+bool forward_tc_supported(const Dims& d, int dtype);
+cudaError_t launch_forward_tc(const Dims& d, const void* Q, const void* K, const void* V,
+                              const float* lce_w, const float* lce_b, void* O, int32_t* index, float* lse,
+                              float* q_mean, float* k_mean, int32_t* ctrl, int32_t* sync, int inject,
+                              cudaStream_t st);
 
 bool attend_img_supported(const Dims& d, int dtype);
 cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
                               const int32_t* index, const float* lce_w, const float* lce_b,
-                              void* O, float* lse, int32_t* status, cudaStream_t st);
+                              void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel);
 bool attend_tc_wide_supported(const Dims& d, int dtype);
 cudaError_t launch_attend_tc_wide(const Dims& d, const void* Q, const void* K, const void* V,
                                   const int32_t* index, const float* lce_w, const float* lce_b,
-                                  void* O, float* lse, int32_t* status, cudaStream_t st);
+                                  void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel);
 
 bool backward_mma_supported(const Dims& d, int dtype);
 cudaError_t launch_backward_mma(const Dims& d, const void* Q, const void* K, const void* V,
@@ -97,22 +105,32 @@ cudaError_t launch_backward_img(const Dims& d, const void* Q, const void* K, con
                                 void* dQ, void* dK, void* dV, float* delta, int32_t* status, cudaStream_t st);
 
 // A process may drive several GPUs, and kernel attributes are per device: the largest value already
-// set for a kernel on the CURRENT device (dynamic shared-memory size, or 1 for "set-up done").
+// set for a kernel on the CURRENT device (dynamic shared-memory size, or 1 for "set-up done").  The
+// set-up runs under a lock and is recorded only once it has succeeded, so concurrent host threads
+// never launch before the attribute exists and a failed set-up is tried again.
 struct PerDeviceMax {
+    std::mutex lock;
     int v[64] = {};
-    // true if `want` exceeds what the current device has been given so far; records it
-    bool raise(int want) {
+    template <typename F>
+    cudaError_t ensure(int want, F&& set) {
         int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
-        if (want <= v[dev]) return false;
-        v[dev] = want;
-        return true;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return set();
+        std::lock_guard<std::mutex> guard(lock);
+        if (want <= v[dev]) return cudaSuccess;
+        const cudaError_t e = set();
+        if (e == cudaSuccess) v[dev] = want;
+        return e;
     }
 };
+struct PerDeviceOnce {
+    PerDeviceMax m;
+    template <typename F>
+    cudaError_t run(F&& set) { return m.ensure(1, set); }
+};
 
-void hint_backward_impl(int impl);     // bra_impl of the call that follows on this thread
 bool backward_supported(const Dims& d);
-cudaError_t launch_backward(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
+// impl: the bra_impl the caller asked for
+cudaError_t launch_backward(const Dims& d, int dtype, int impl, const void* Q, const void* K, const void* V,
                             const int32_t* index, const float* lce_w, const float* lse,
                             const void* dO, void* dQ, void* dK, void* dV,
                             float* d_lce_w, float* d_lce_b,

@@ -19,6 +19,9 @@ pytestmark = pytest.mark.gpu
 
 TOL = {"bf16": dict(max=2e-2, mean=2e-3), "f32": dict(max=1e-5, mean=1e-6)}
 GRAD_MAX = 5e-2
+# d_lce_w / d_lce_b are sums over all B*H*W positions of products that are exact in fp32; with
+# fp32 partial sums the rounding error is about sqrt(n) * 2^-24 of the running sum (n <= 2e5 here)
+LCE_GRAD_REL = 1e-4
 
 
 @pytest.fixture(scope="module")
@@ -161,6 +164,10 @@ IMPLS = {"simt": 1, "mma": 2, "tc": 3, "img": 4, "auto": 0}
 
 def run_attend_case(bra, cfg, impl, seed, shared=False, lce=True, bias=False, scale=0.0,
                     index=None, clustered=False):
+    """One bra_attend call of kernel family `impl` against the oracle.  A family that is
+    named explicitly must take the shape: BRA_ERR_UNSUPPORTED fails the test (the cases
+    where a family rightly refuses a shape are asserted in
+    test_kernel_families_refuse_only_what_they_should)."""
     import torch
     x = synthetic.make_inputs(cfg, seed=seed, clustered=clustered)
     t = to_dev(x, cfg)
@@ -175,12 +182,7 @@ def run_attend_case(bra, cfg, impl, seed, shared=False, lce=True, bias=False, sc
     if bias:
         b_np = np.linspace(-0.5, 0.5, cfg.C).astype(np.float32)
         b = torch.from_numpy(b_np).cuda()
-    try:
-        O, lse = bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"] if lce else None, b, ws=ws)
-    except bra.BraError as e:
-        if e.code == 7 and impl != "simt":
-            pytest.skip(f"{impl} kernel does not take {cfg.name}")
-        raise
+    O, lse = bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"] if lce else None, b, ws=ws)
     assert bra.last_launch_count() >= 1
     assert bra.bra_device_status(ws) == 0
     O_ref, lse_ref = orc.bra_attend(x["Q"], x["K"], x["V"], idx.cpu().numpy(),
@@ -191,10 +193,32 @@ def run_attend_case(bra, cfg, impl, seed, shared=False, lce=True, bias=False, sc
     return O
 
 
-@pytest.mark.parametrize("impl", ["simt", "mma", "tc", "img", "auto"])
-@pytest.mark.parametrize("n", [1, 2, 3, 4, 5])
+# which benchmark configs each kernel family takes: fp32 (config 1) only the CUDA-core kernel;
+# tcgen05 wants 8 x 8 or 16-wide regions (configs 2, 4); the image-resident kernel wants a head's
+# K and V of a whole image in shared memory (configs 3, 5)
+TAKES = {"simt": {1, 2, 3, 4, 5}, "mma": {2, 3, 4, 5}, "tc": {2, 4}, "img": {3, 5}, "auto": {1, 2, 3, 4, 5}}
+
+
+@pytest.mark.parametrize("impl,n", [(i, n) for i in TAKES for n in sorted(TAKES[i])])
 def test_attend_matches_oracle_on_benchmark_configs(bra, n, impl):
     run_attend_case(bra, CONFIGS[n], impl, seed=1000 + n)
+
+
+@pytest.mark.parametrize("impl,n", [(i, n) for i in TAKES for n in range(1, 6) if n not in TAKES[i]])
+def test_kernel_families_refuse_only_what_they_should(bra, n, impl):
+    """A family asked for a shape outside its range answers BRA_ERR_UNSUPPORTED on the host,
+    nothing launched; every other (family, config) pair is a parity case above."""
+    import torch
+    cfg = CONFIGS[n]
+    x = synthetic.make_inputs(synthetic.with_batch(cfg, 1), seed=3)
+    small = synthetic.with_batch(cfg, 1)
+    t = to_dev(x, small)
+    p = problem_of(bra, small, impl=IMPLS[impl])
+    idx = torch.zeros(1, small.heads, small.R, small.topk, dtype=torch.int32, device="cuda")
+    with pytest.raises(bra.BraError) as e:
+        bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"])
+    assert e.value.code == 7
+    assert bra.last_launch_count() == 0
 
 
 EDGE = [
@@ -414,6 +438,87 @@ def test_forward_orders_attention_after_routing(bra, n):
         assert (idx == idx_ref).all() and (O == O_ref).all(), f"call {it}"
 
 
+# bf16, head dim 32, 8 x 8-token regions, topk = 1, per-head routing, <= 64 regions, C <= 128:
+# bra_forward is ONE kernel launch (pooling, routing and attention as numbered jobs of one grid)
+ONE_LAUNCH_CASES = [
+    BraConfig("fused-single-region", 1, 8, 8, 64, 2, 1, 1, "bf16"),
+    BraConfig("fused-one-image", 1, 56, 56, 64, 2, 7, 1, "bf16"),
+    BraConfig("fused-two-head-pairs", 3, 32, 32, 128, 4, 4, 1, "bf16"),
+    BraConfig("fused-64-regions", 2, 64, 64, 64, 2, 8, 1, "bf16"),
+    BraConfig("fused-nine-regions", 5, 24, 24, 64, 2, 3, 1, "bf16"),
+    BraConfig("fused-more-images-than-lookahead", 40, 16, 16, 64, 2, 2, 1, "bf16"),
+]
+
+
+@pytest.mark.parametrize("cfg", ONE_LAUNCH_CASES, ids=[c.name for c in ONE_LAUNCH_CASES])
+def test_forward_in_one_launch_equals_route_then_attend(bra, cfg):
+    """The one-launch forward gives, bit for bit, the index of bra_route and the O / lse of bra_attend,
+    call after call on the same scratch buffer (its counters and flags clean themselves), and matches
+    the oracle."""
+    import torch
+    p = problem_of(bra, cfg)
+    ws = bra.workspace(p)
+    sets = [to_dev(synthetic.make_inputs(cfg, seed=300 + s, clustered=bool(s)), cfg) for s in range(2)]
+    want = []
+    for t in sets:
+        _, _, idx = bra.bra_route(p, t["Q"], t["K"], ws=ws)
+        O, lse = bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"], ws=ws)
+        want.append((idx.clone(), O.clone(), lse.clone()))
+    for it in range(5):
+        t, (idx_ref, O_ref, lse_ref) = sets[it % 2], want[it % 2]
+        O, idx, lse = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+        assert bra.last_launch_count() == 1
+        assert bra.bra_device_status(ws) == 0, f"call {it}"
+        assert (idx == idx_ref).all(), f"call {it}"
+        assert (O == O_ref).all() and (lse == lse_ref).all(), f"call {it}"
+    x = synthetic.make_inputs(cfg, seed=300)
+    _, _, idx_o, gap = orc.bra_route(x["Q"], x["K"], cfg.heads, cfg.S, cfg.topk)
+    check_index(want[0][0].cpu().numpy(), idx_o, gap, cfg.topk, cfg.R, oracle_affinity(x, cfg))
+    O_o, _ = orc.bra_attend(x["Q"], x["K"], x["V"], want[0][0].cpu().numpy(), x["w"], cfg.heads, cfg.S)
+    check_O(f64(want[0][1]), O_o, cfg.dtype)
+
+
+def test_bounded_wait_that_runs_out_is_reported_and_recoverable(bra):
+    """Failure detection without a GPU fault: with the injection switch the routing step of the
+    one-launch forward never raises its per-image flags, so the attention jobs' bounded waits run
+    out (nothing is in flight on the tensor cores at that point), the kernel returns, and the status
+    reads BRA_ERR_TIMEOUT.  Reading the status restores the scratch buffer: the next call is clean."""
+    cfg = BraConfig("timeout", 3, 32, 32, 64, 2, 4, 1, "bf16")
+    t = to_dev(synthetic.make_inputs(cfg, seed=9), cfg)
+    p = problem_of(bra, cfg)
+    ws = bra.workspace(p)
+    O_ref, idx_ref, _ = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+    assert bra.bra_device_status(ws) == 0
+    p_bad = problem_of(bra, cfg, inject=1)
+    bra.bra_forward(p_bad, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+    assert bra.bra_device_status(ws) == 10
+    assert bra.bra_device_status(ws) == 0          # cleared by the read
+    for _ in range(2):
+        O, idx, _ = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+        assert bra.bra_device_status(ws) == 0
+        assert (O == O_ref).all() and (idx == idx_ref).all()
+
+
+def test_workspace_init_makes_a_dirty_buffer_usable(bra):
+    """A scratch buffer full of garbage: after bra_workspace_init an out-of-range index entry is still
+    reported, and the one-launch forward (which needs its counters at zero) gives the right result."""
+    import torch
+    cfg = BraConfig("dirty-ws", 2, 32, 32, 64, 2, 4, 1, "bf16")
+    t = to_dev(synthetic.make_inputs(cfg, seed=10), cfg)
+    p = problem_of(bra, cfg)
+    O_ref, idx_ref, _ = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"])
+    ws = bra.workspace(p)
+    ws.fill_(0xFF)
+    bra.workspace_init(p, ws)
+    bad = idx_ref.clone()
+    bad[1, 0, 3, 0] = cfg.R
+    bra.bra_attend(p, t["Q"], t["K"], t["V"], bad, t["w"], ws=ws)
+    assert bra.bra_device_status(ws) == 9
+    O, idx, _ = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+    assert bra.bra_device_status(ws) == 0
+    assert (O == O_ref).all() and (idx == idx_ref).all()
+
+
 # ------------------------------------------------------------------ backward
 def run_backward_case(bra, cfg, seed, clustered=False, shared=False, index=None, impl="auto"):
     import torch
@@ -437,8 +542,11 @@ def run_backward_case(bra, cfg, seed, clustered=False, shared=False, index=None,
     tol = GRAD_MAX if cfg.dtype == "bf16" else 2e-4
     for name, g, r in zip(names, g1, ref):
         err = np.abs(f64(g) - r).max()
-        scale = max(1.0, np.abs(r).max()) if name.startswith("d_lce") else 1.0
-        assert err <= tol * scale, f"{cfg.name} {name}: max-abs {err:.3e}"
+        assert err <= tol, f"{cfg.name} {name}: max-abs {err:.3e}"
+        if name.startswith("d_lce"):
+            # sums of B*H*W exact products accumulated in fp32: besides the stated absolute
+            # bound, the error stays a small fraction of the largest entry
+            assert err <= LCE_GRAD_REL * max(1.0, np.abs(r).max()), f"{cfg.name} {name}: {err:.3e} rel"
 
 
 def test_backward_tiny_fp32(bra):
@@ -546,7 +654,6 @@ def test_random_shapes_forward_and_backward(bra, seed):
         assert bra.bra_device_status(ws_buf) == 0
         ref = orc.bra_backward(x["Q"], x["K"], x["V"], idn, x["w"], x["dO"], cfg.heads, cfg.S)
         for name, a, r in zip(("dQ", "dK", "dV", "d_lce_w", "d_lce_b"), g, ref):
-            scale = max(1.0, np.abs(r).max()) if name.startswith("d_lce") else 1.0
-            assert np.abs(f64(a) - r).max() <= GRAD_MAX * scale, f"{cfg} {impl} {name}"
+            assert np.abs(f64(a) - r).max() <= GRAD_MAX, f"{cfg} {impl} {name}"
         ran += 1
     assert ran >= 8

@@ -449,17 +449,77 @@ def test_backward_full_attention_case_matches_textbook_gradient():
 
 
 # ---------------------------------------------------------------- planted mistakes
-def test_pins_catch_planted_mistakes(monkeypatch):
-    """A dropped scale, a flipped LCE kernel or a sum instead of a mean in the
-    oracle must break a pin (run a pin against a sabotaged copy)."""
-    Q, K, V = small_problem(31, H=8, W=8)
-    w = rng(32).standard_normal((4, 5, 5))
-    good = orc.lce(V, w)
-    flipped = orc.lce(V, w[:, ::-1, ::-1])
-    assert not np.allclose(good, flipped)
-    Of, _ = full_attention_loops(Q, K, V, 2, 0.37)
-    O_noscale, *_ = orc.bra_forward(Q, K, V, None, 2, 2, 4, scale=1.0)
-    assert not np.allclose(Of, O_noscale)
-    # a sum in place of the mean changes the affinity by n_r^2
-    Qr = orc.region_means(Q, 2)
-    assert np.allclose(Qr * 16, orc.region_partition(Q, 2).sum(axis=2))
+def _sum_for_mean(X, S):
+    return orc.region_partition(np.asarray(X, dtype=np.float64), S).sum(axis=2)
+
+
+def _transposed_affinity(real):
+    def f(Qr, Kr, heads, shared_routing=False):
+        return real(Kr, Qr, heads, shared_routing)
+    return f
+
+
+def _ties_to_higher_index(real):
+    def f(A, k):
+        idx, gap = real(A[..., ::-1], k)
+        return (A.shape[-1] - 1 - idx).astype(np.int32), gap
+    return f
+
+
+def _no_max_subtraction_wrong_sign(real):
+    def f(Q, K, V, index, heads, S, scale):
+        return real(Q, K, V, index, heads, S, -scale)
+    return f
+
+
+def _flipped_filter(real):
+    def f(V, w, bias=None):
+        return real(V, np.asarray(w)[:, ::-1, ::-1], bias)
+    return f
+
+
+def _replicated_border(real):
+    def f(V, w, bias=None):
+        V = np.asarray(V, dtype=np.float64)
+        big = np.pad(V, ((0, 0), (2, 2), (2, 2), (0, 0)), mode="edge")   # edge values, not zeros, outside the map
+        return real(big, w, bias)[:, 2:-2, 2:-2]
+    return f
+
+
+def _wrong_scale(C, heads):
+    return 1.0 / np.sqrt(C)
+
+
+def _dropped_lce_adjoint(real):
+    def f(Q, K, V, index, w, dO, heads, S, scale=None):
+        return real(Q, K, V, index, np.zeros_like(np.asarray(w, dtype=np.float64)), dO, heads, S, scale)
+    return f
+
+
+PLANTED = [
+    # (oracle attribute, sabotage, pins of which at least the first must fail)
+    ("region_means", lambda real: _sum_for_mean, ["test_affinity_is_mean_of_all_token_pair_products"]),
+    ("region_affinity", _transposed_affinity, ["test_affinity_is_mean_of_all_token_pair_products"]),
+    ("topk_index", _ties_to_higher_index, ["test_topk_tie_break_lower_index_first"]),
+    ("routed_attention", _no_max_subtraction_wrong_sign, ["test_topk_equal_S2_is_full_attention",
+                                                          "test_S1_is_full_attention"]),
+    ("default_scale", lambda real: _wrong_scale, ["test_default_scale_is_one_over_sqrt_head_dim"]),
+    ("lce", _flipped_filter, ["test_lce_shifted_delta_picks_the_right_neighbour",
+                              "test_lce_matches_scipy_correlate2d"]),
+    ("lce", _replicated_border, ["test_lce_all_ones_border_sums_by_hand",
+                                  "test_lce_matches_scipy_correlate2d"]),
+    ("bra_backward", _dropped_lce_adjoint, ["test_backward_matches_central_finite_differences"]),
+]
+
+
+@pytest.mark.parametrize("attr,sabotage,pins", PLANTED, ids=[f"{a}-{i}" for i, (a, _, _) in enumerate(PLANTED)])
+def test_pins_catch_planted_mistakes(monkeypatch, attr, sabotage, pins):
+    """Plant one mistake in the oracle (a sum for the mean, a transposed operand, the wrong
+    tie-break, a sign, the wrong scale, a flipped filter, a border that is not zero, a
+    dropped gradient term) and run the named pins against the sabotaged oracle: each must fail."""
+    for name in pins:
+        globals()[name]()                               # green on the oracle as it stands
+    monkeypatch.setattr(orc, attr, sabotage(getattr(orc, attr)))
+    for name in pins:
+        with pytest.raises((AssertionError, IndexError, ValueError)):
+            globals()[name]()
