@@ -70,14 +70,17 @@ typedef enum bra_impl {
     BRA_IMPL_SIMT = 1,  /* fp32 CUDA-core kernel: any dtype, any shape with C/heads <= 128 */
     BRA_IMPL_MMA = 2,   /* bf16 warp-level tensor-core kernel (C/heads == 32) */
     BRA_IMPL_TC = 3,    /* bf16 tcgen05/TMEM kernels (C/heads == 32; regions of 8 x 8 tokens, or 16 wide and a multiple of 8 high) */
-    BRA_IMPL_IMG = 4    /* bf16 warp-level tensor-core kernel with a whole (image, head) of K and V resident in
+    BRA_IMPL_IMG = 4,   /* bf16 warp-level tensor-core kernel with a whole (image, head) of K and V resident in
                            shared memory (C/heads == 32, H*W <= ~1500 tokens): small maps, small regions */
+    BRA_IMPL_TC_FUSED = 5 /* as BRA_IMPL_TC, and bra_forward runs pooling, routing and attention in ONE launch
+                           (8 x 8-token regions, topk = 1, per-head routing, <= 64 regions, C <= 128); never
+                           chosen by BRA_IMPL_AUTO: on B200 the chain of three launches is faster */
 } bra_impl;
 
 /*
  * Failure injection for tests of the error path (no GPU fault, trap or hang is involved).
- * BRA_INJECT_HOLD_ROUTE_FLAGS: in the one-launch forward (bra_forward on 8 x 8-token regions with
- * topk = 1) the routing step keeps the per-image "routed" flags down, so every attention job's bounded
+ * BRA_INJECT_HOLD_ROUTE_FLAGS: in the one-launch forward (bra_forward with BRA_IMPL_TC_FUSED) the
+ * routing step keeps the per-image "routed" flags down, so every attention job's bounded
  * wait on them runs out after a few thousand polls with no tensor-core work in flight; the kernel returns
  * normally, O is not written and bra_device_status() reports BRA_ERR_TIMEOUT.  Ignored by every other path.
  */
@@ -173,9 +176,8 @@ bra_status bra_attend(const bra_problem* p, const void* Q, const void* K, const 
 
 /*
  * Algorithm 1 from the projected Q, K, V on: bra_route then bra_attend in one call; same results,
- * bit for bit, as the two calls.  For bf16 problems with head dim 32, 8 x 8-token regions, topk = 1,
- * per-head routing, at most 64 regions and C <= 128 the whole call is ONE kernel launch (pooling,
- * Eq. 4, Eq. 5 and the attention overlap inside it); other problems chain the library's kernels.
+ * bit for bit, as the two calls.  The library's kernels are chained on `stream` and overlap at their
+ * ends; with BRA_IMPL_TC_FUSED the whole call is one kernel launch.
  *   index    out  may be NULL (then kept in ws only)
  *   lse      out  may be NULL
  */

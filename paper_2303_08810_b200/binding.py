@@ -14,7 +14,7 @@ from ctypes import c_float, c_int32, c_size_t, c_void_p
 _LIB = None
 _LIB_NAME = "libbra_b200.so"
 
-IMPL_AUTO, IMPL_SIMT, IMPL_MMA, IMPL_TC, IMPL_IMG = 0, 1, 2, 3, 4
+IMPL_AUTO, IMPL_SIMT, IMPL_MMA, IMPL_TC, IMPL_IMG, IMPL_TC_FUSED = 0, 1, 2, 3, 4, 5
 F32, BF16 = 0, 1
 
 

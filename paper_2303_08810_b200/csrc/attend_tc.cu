@@ -1,6 +1,6 @@
 // Routed token-to-token attention + LCE on the 5th-generation tensor cores
-// (Eq. 6, Eq. 7 with Eq. 1), and the whole forward pass of Algorithm 1 in ONE launch
-// (region pooling, Eq. 4, Eq. 5, then the attention) for the same shapes.
+// (Eq. 6, Eq. 7 with Eq. 1) for any topk: the kernel for topk >= 2; topk = 1 has a kernel
+// of its own (attend_tc_k1.cu) that shares this file's tile layout.
 //
 // Shape handled here: head dim 32, regions of 8 x 8 = 64 tokens, heads in pairs.
 // A tile is (image b, query region i, head pair hp) = 64 tokens x 64 channels of O.
@@ -12,271 +12,45 @@
 // and V is 64 x 64 with key j's row = (head A's channels of token j of A's region | head
 // B's channels of token j of B's region); each row then keeps its own head's 32 columns.
 //
-// Small CTAs (128 threads, ~52 KB of shared memory, 128 TMEM columns), four per SM,
-// each walking its own tiles start to finish; the SM overlaps the CTAs' phases.
-// Measured on this shape, that beats one large warp-specialised CTA per SM: the work
-// per tile is too small to pay for hand-offs between specialised warps.  Per tile:
+// Small CTAs (128 threads, ~70 KB of shared memory, 128 TMEM columns), three per SM,
+// each walking its own tiles start to finish; the SM overlaps the CTAs' phases.  Per tile:
 //   1. all threads: 16-byte cp.async copies of the Q tile, of the K and V tiles of the
 //      routed regions (K^g / V^g are never formed in HBM: the routing index only picks
 //      the source addresses) and of the 12 x 12 V halo, written in the swizzled layouts
-//      the MMA descriptors name.  Q and K of the next tile go out as soon as the last
-//      MMA of the tile in hand has read its operands, V and the halo after its LCE.
+//      the MMA descriptors name.  K/V of routed step m + 1 stream into the other buffer
+//      during step m; Q and K of the next tile go out as soon as the last MMA of the tile
+//      in hand has read its operands, V and the halo after its LCE.
 //   2. one thread: tcgen05.mma S = Q K^T into TMEM (fp32)
-//   3. thread = row: softmax; P (bf16 pairs) overwrites S in TMEM columns 0..63
-//   4. one thread: tcgen05.mma O = P V with P read from TMEM; O lands in columns 64..95
+//   3. thread = row: online softmax; P (bf16 pairs) overwrites S in TMEM columns 0..63
+//   4. one thread: tcgen05.mma P V with P read from TMEM; lands in columns 64..95 and is
+//      folded into the running O in registers
 //   5. thread = row: normalised O^att to an fp32 staging tile
 //   6. warp = 2 columns of the region, lane = channel pair: LCE, the 5x5 depthwise
 //      correlation of V from the halo tile with the weights in registers, on top of
 //      O^att, one bf16 store of O.
-//
-// Fused forward (template parameter FUSED): the CTAs draw numbered jobs from a counter.
-// Job t = (image slot s, unit u = (region, head pair)) pools unit u of image s (the
-// per-region average of Q and K, summed in the order of the stand-alone pooling kernel)
-// and attends unit u of image s - delta.  The CTA that completes an image's pooling also
-// routes it (Eq. 4 and Eq. 5 for every region and head, in the order of the stand-alone
-// routing kernels: the index is bit-identical) and raises the image's flag; attention
-// jobs wait on that flag.  delta is chosen so that, in the steady state, the flag was
-// raised long before it is looked at.  A wait only ever depends on jobs with smaller
-// numbers, and a job's pooling part never waits, so the scheme cannot deadlock whatever
-// the number of resident CTAs; every wait is bounded all the same.
 // Hot loops are kept rolled and short (straight-line per-tile code was bound by
 // instruction fetch).  Every wait on an MMA is bounded.
-#include "bra_internal.h"
-#include "sm100_ptx.cuh"
+#include "attend_tc_common.cuh"
 
 namespace bra {
 
-using namespace ptx;
-
-namespace tc {
-constexpr int RS = 8;            // region side in tokens
-constexpr int HALO = RS + 4;     // 12: region plus the 2-token LCE border
-constexpr int THREADS = 128;
-constexpr int KCAP = 64;         // largest topk
-constexpr int TMEM_COLS = 128;   // S [0,128) fp32; then P [0,32) bf16 pairs + O [64,128)
-constexpr int TM_O = 64;
-constexpr int HALO_BYTES = HALO * HALO * 128;            // 18432
-// shared memory map (bytes, from a 1024-byte aligned base)
-constexpr int OFF_Q = 0;                                 // [128 rows][64 B]  64B swizzle, K-major
-constexpr int OFF_K = 8192;                              // [128 keys][64 B]  64B swizzle, K-major (buffer 0)
-constexpr int OFF_V = 16384;                             // [64 keys][128 B]  128B swizzle, MN-major (buffer 0)
-constexpr int OFF_ST = OFF_V;                            // [64 tokens][64 ch] fp32 staging: over V (buffer 0) + scratch
-constexpr int OFF_POOL = 24576;                          // 8 KB scratch of the fused forward: pooling partial sums, K^r of a head
-constexpr int OFF_HALO = 32768;                          // [12][12][64 ch] bf16, linear
-constexpr int OFF_BAR = OFF_HALO + HALO_BYTES;           // 51200: two mbarriers, tmem slot, job slots
-constexpr int OFF_MISC = OFF_BAR + 64;                   // 1 KB: routing step, best key per (half, row)
-constexpr int OFF_KV1 = 53248;                           // topk > 1 only: K buffer 1 (8 KB), V buffer 1 (8 KB)
-constexpr int SMEM_K1 = OFF_MISC + 1024 + 1024;          // + slack for the manual 1024-byte alignment
-constexpr int SMEM_KN = OFF_KV1 + 16384 + 1024;
-static_assert(OFF_KV1 % 1024 == 0 && OFF_KV1 >= OFF_MISC + 1024, "buffer 1 placement");
-constexpr uint32_t POLL_LIMIT = 4000000u;
-constexpr uint32_t FLAG_POLLS = 1u << 20;                // x ~0.1-0.5 us per poll: a fraction of a second
-constexpr int FUSED_MAX_R = 64;                          // routing step: one thread per (row, half of the candidates)
-}  // namespace tc
-
-__device__ __forceinline__ float ex2f(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&h);
-}
-__device__ __forceinline__ uint4 ldg_nc_u4(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
-__device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t* p) {
-    int32_t v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_release_gpu(int32_t* p, int32_t v) {
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-// order-preserving bits of an fp32 score (-0 and +0 tie), as in the stand-alone routing kernels
-__device__ __forceinline__ uint32_t score_bits(float s) {
-    s += 0.0f;
-    const uint32_t u = __float_as_uint(s);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
-#ifdef BRA_EXP_TRACE
-__device__ long long g_trace[4 * 16 * 10];
-__device__ int g_trace_cnt[16];
-#define BRA_TR(n, ev)                                                                                   \
-    do {                                                                                                \
-        if (threadIdx.x == 0 && (blockIdx.x & 127) == 0 && blockIdx.x < 512 && (n) < 16)                  \
-            g_trace[((blockIdx.x >> 7) * 16 + (n)) * 10 + (ev)] = clock64();                             \
-    } while (0)
-#define BRA_CNT(i, v) do { if (threadIdx.x == 0) atomicAdd(&g_trace_cnt[i], (int)(v)); } while (0)
-#else
-#define BRA_TR(n, ev) do { } while (0)
-#define BRA_CNT(i, v) do { } while (0)
-#endif
-
-struct TileCoord { int b, i, hp, y0, x0, c0; };
-// Walks tiles T, T + stride, ... (T = (b * R + i) * pairs + hp) with adds and carries only.
-struct TileWalker {
-    int pairs, R;
-    int d_hp, d_i, d_b;                // stride split into (hp, i, b) digits
-    int hp, i, b;
-    __device__ __forceinline__ void init(int T, int stride, const Dims& dm) {
-        pairs = dm.heads >> 1; R = dm.R;
-        hp = T % pairs; i = (T / pairs) % R; b = T / (pairs * R);
-        d_hp = stride % pairs; d_i = (stride / pairs) % R; d_b = stride / (pairs * R);
-    }
-    __device__ __forceinline__ void next() {
-        hp += d_hp;
-        int carry = hp >= pairs;
-        hp -= carry ? pairs : 0;
-        i += d_i + carry;
-        carry = i >= R;
-        i -= carry ? R : 0;
-        b += d_b + carry;
-    }
-};
-
-// What the fused forward adds to the arguments of the attention kernel.
-struct FusedArgs {
-    float* q_mean;          // [B,R,C] Q^r (scratch)
-    float* k_mean;          // [B,R,C] K^r (scratch)
-    int32_t* index_out;     // [B,heads,R,1] written by the routing step, read by the attention part
-    int32_t* pool_cnt;      // [B] units of image b pooled so far        } zero at launch,
-    int32_t* route_flag;    // [B] 1 once the index of image b is written  } zeroed again by the last CTA
-    int32_t* ctrl;          // status block: [8] job counter, [9] finished CTAs (same rule)
-    int delta;              // images the pooling runs ahead of the attention
-    int units;              // R * head pairs: jobs per image slot
-    int total;              // (B + delta) * units jobs
-    int inject;             // failure injection of the tests: 1 = the flags are never raised
-    int sync_off, sync_bytes;   // where pool_cnt / route_flag sit in the scratch buffer (recorded in ctrl[2], ctrl[3])
-};
-struct Job { int att_b, pool_b, i, hp; };      // image of the attention / pooling part (-1: none), region, head pair
-
-// Fused forward: Eq. 4 + Eq. 5 (k = 1) for every region and head of image b, by the whole CTA; then the
-// image's flag goes up.  Kept out of line: it runs once per image and must not weigh on the register
-// allocation of the tile loop.
-__device__ __noinline__ void route_image(const FusedArgs& fa, const Dims& dm, int b, uint8_t* smem) {
-    using namespace tc;
-    const int tid = threadIdx.x;
-    const uint32_t sm_base = smem_u32(smem);
-    // K^r of one head sits in the 8 KB scratch as [R][8 x 16 B], unit (c4 + j) & 7 of row j holding channels 4 c4..4 c4+3 (conflict-free
-    // for 16-byte reads by consecutive rows); thread = (row i, half of the candidates), four candidates
-    // at a time (independent chains; each dot product adds its channels in increasing order).
-    const uint32_t ks = sm_base + OFF_POOL;
-    unsigned long long* best_slot = reinterpret_cast<unsigned long long*>(smem + OFF_MISC);
-    const int i = tid & 63, half = tid >> 6;
-    const int jmid = (dm.R + 1) >> 1;
-    const int j0 = half ? jmid : 0, j1 = half ? dm.R : jmid;
-    const int nchunk = dm.R * 8;
-    float4 kst[4];                                   // this thread's part of K^r of the head to come
-    auto fetch_k = [&](int h) {
-        const float* kb = fa.k_mean + (size_t)b * dm.R * dm.C + h * 32;
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int e = tid + u * THREADS;
-            if (e < nchunk) kst[u] = __ldcg(reinterpret_cast<const float4*>(kb + (size_t)(e >> 3) * dm.C) + (e & 7));
-        }
-    };
-    fetch_k(0);
-#ifdef BRA_EXP_TRACE
-    long long rt0 = clock64();
-#endif
-    for (int h = 0; h < dm.heads; ++h) {
-        float4 q[8];
-        if (i < dm.R) {
-            const float4* qrow = reinterpret_cast<const float4*>(fa.q_mean + ((size_t)b * dm.R + i) * dm.C + h * 32);
-#pragma unroll
-            for (int c4 = 0; c4 < 8; ++c4) q[c4] = __ldcg(qrow + c4);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int e = tid + u * THREADS;
-            const int j = e >> 3, c4 = e & 7;
-            if (e < nchunk) sts_f32x4(ks + ((j * 8 + ((c4 + j) & 7)) << 4), kst[u].x, kst[u].y, kst[u].z, kst[u].w);
-        }
-        __syncthreads();
-#ifdef BRA_EXP_TRACE
-        if (h == 0) BRA_CNT(5, (clock64() - rt0) >> 4);
-#endif
-        if (h + 1 < dm.heads) fetch_k(h + 1);
-        if (i < dm.R) {
-            unsigned long long best = 0ull;
-            for (int j = j0; j < j1; j += 4) {
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                int jj[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) jj[e] = j + e < j1 ? j + e : j1 - 1;
-#pragma unroll
-                for (int c4 = 0; c4 < 8; ++c4) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float4 k4 = lds_f32x4(ks + ((jj[e] * 8 + ((c4 + jj[e]) & 7)) << 4));
-                        acc[e] = fmaf(q[c4].x, k4.x, acc[e]);
-                        acc[e] = fmaf(q[c4].y, k4.y, acc[e]);
-                        acc[e] = fmaf(q[c4].z, k4.z, acc[e]);
-                        acc[e] = fmaf(q[c4].w, k4.w, acc[e]);
-                    }
-                }
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {        // a clamped repeat of the last candidate changes nothing
-                    const unsigned long long key = ((unsigned long long)score_bits(acc[e]) << 32) | (0xffffffffu - (uint32_t)jj[e]);
-                    best = key > best ? key : best;
-                }
-            }
-            best_slot[half * 64 + i] = best;
-        }
-#ifdef BRA_EXP_TRACE
-        if (h == 0) BRA_CNT(6, (clock64() - rt0) >> 4);
-#endif
-        __syncthreads();
-#ifdef BRA_EXP_TRACE
-        if (h == 0) BRA_CNT(7, (clock64() - rt0) >> 4);
-#endif
-        if (tid < dm.R) {
-            const unsigned long long a = best_slot[tid], bb = best_slot[64 + tid];
-            const unsigned long long top = a > bb ? a : bb;
-            fa.index_out[((size_t)b * dm.heads + h) * dm.R + tid] = (int32_t)(0xffffffffu - (uint32_t)top);
-        }
-        // (the scratch is rewritten only after this barrier, best_slot only after the next head's first one)
-    }
-#ifdef BRA_EXP_TRACE
-    BRA_CNT(8, (clock64() - rt0) >> 4);
-#endif
-    __threadfence();
-    __syncthreads();
-#ifdef BRA_EXP_TRACE
-    BRA_CNT(9, (clock64() - rt0) >> 4);
-#endif
-    if (tid == 0 && !fa.inject) st_release_gpu(fa.route_flag + b, 1);
-}
-
-// K1: topk == 1 (one routed step per tile: no running maximum, no rescaling of O, one K/V buffer).
-// FUSED: the forward pass in one launch (see the head of the file); needs K1.
-template <bool K1, bool FUSED>
-__global__ void __launch_bounds__(tc::THREADS, K1 ? 4 : 3)
+__global__ void __launch_bounds__(tc::THREADS, 3)
 attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
                  const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
                  const float* __restrict__ lce_w, const float* __restrict__ lce_b,
                  __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
-                 int32_t* __restrict__ status, Dims dm, int num_tiles, FusedArgs fa) {
+                 int32_t* __restrict__ status, Dims dm, int num_tiles) {
     using namespace tc;
-    static_assert(!FUSED || K1, "the fused forward is built for topk == 1");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem + OFF_BAR);       // S landed in TMEM
     uint64_t* bar_o = bar_s + 1;                                         // O landed in TMEM
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_s + 2);
-    int* last_slot = reinterpret_cast<int*>(tmem_slot + 1);              // fused: "this CTA routes the image"
-    int4* job_slot = reinterpret_cast<int4*>(smem + OFF_BAR + 32);       // fused: two decoded jobs
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int k = K1 ? 1 : dm.topk;
-    const int pairs = dm.heads >> 1;
+    const int k = dm.topk;
     const int inv_s = (1 << 20) / dm.S + 1;            // i / S == (i * inv_s) >> 20 for i < 4096
+    const int my_tiles = (num_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
 
     if (tid == 0) {
         mbar_init(bar_s, 1);
@@ -288,6 +62,8 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
+    TileWalker walk;
+    walk.init(blockIdx.x, gridDim.x, dm);
 
     // ---- loader mapping: thread copies 16-byte chunk c of the 128-byte channel row (both
     // heads) of token column tx, in token rows lrow..lrow+3 of a region: a warp covers 512
@@ -315,19 +91,16 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
     const uint32_t o_addr = tg + TM_O + head_half * 32;   // this row's 32 channels of O
     const float sl2 = dm.scale * 1.4426950408889634f;
     // ---- LCE mapping: warp = 2 columns of the region, lane = channel pair
-    // The weights of a channel pair stay in registers from tile to tile; the fused forward, which needs
-    // the registers for the pooling loads in flight, fetches them again (cache hits) before each LCE.
     const int xl0 = 2 * warp;
-    float2 wv_keep[25];
+    float2 wv[25];
 #pragma unroll
-    for (int q = 0; q < 25; ++q) wv_keep[q] = make_float2(0.f, 0.f);
-    float2 bias_keep = make_float2(0.f, 0.f);
+    for (int q = 0; q < 25; ++q) wv[q] = make_float2(0.f, 0.f);
+    float2 bias2 = make_float2(0.f, 0.f);
     int hp_loaded = -1;
 
     constexpr uint32_t IDESC_S = umma_idesc_bf16(128, 128, false, false);
     constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 64, false, true);
 
-    bool ok = true;
     auto coord_of = [&](int b, int i, int hp) -> TileCoord {
         TileCoord t;
         t.b = b; t.i = i; t.hp = hp;
@@ -343,36 +116,16 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
         return (size_t)b * img_bytes + (size_t)(ry * RS) * row_bytes + (size_t)(rx * RS) * dm.C * 2 + (size_t)c0 * 2 + thr_off;
     };
     // routing entries (head A, head B) of a unit = (tile, routed step); -1: out of range.  The index may
-    // come from a kernel this one overlaps (programmatic dependent launch) or, in the fused forward,
-    // from another CTA of this launch: coherent loads after the wait, never the read-only path
-    auto index_entries = [&](const TileCoord& t, int m) -> int2 {
+    // come from a kernel this one overlaps (programmatic dependent launch): coherent loads after
+    // pdl_wait(), never the read-only path, whose loads the compiler may move above the wait
+    auto read_entries = [&](const TileCoord& t, int m) -> int2 {
         const int hA = 2 * t.hp, hB = hA + 1;
         const int hiA = dm.heads_i == 1 ? 0 : hA, hiB = dm.heads_i == 1 ? 0 : hB;
         int ra = __ldcg(index + (((size_t)t.b * dm.heads_i + hiA) * dm.R + t.i) * dm.topk + m);
         int rb = __ldcg(index + (((size_t)t.b * dm.heads_i + hiB) * dm.R + t.i) * dm.topk + m);
+        if (ra < 0 || ra >= dm.R) { record_error(status, BRA_ERR_INDEX, ra); ra = -1; }
+        if (rb < 0 || rb >= dm.R) { record_error(status, BRA_ERR_INDEX, rb); rb = -1; }
         return make_int2(ra, rb);
-    };
-    auto checked = [&](int2 e) -> int2 {
-        if (e.x < 0 || e.x >= dm.R) { record_error(status, BRA_ERR_INDEX, e.x); e.x = -1; }
-        if (e.y < 0 || e.y >= dm.R) { record_error(status, BRA_ERR_INDEX, e.y); e.y = -1; }
-        return e;
-    };
-    // fused forward: bounded wait until the image of tile t has been routed
-    auto wait_routed = [&](const TileCoord& t) -> bool {
-        const int32_t* flag = fa.route_flag + t.b;
-        const uint32_t limit = fa.inject ? 2048u : FLAG_POLLS;
-        for (uint32_t it = 0; it < limit; ++it) {
-            if (ld_acquire_gpu(flag) != 0) return true;
-            __nanosleep(it < 64 ? 32 : 256);
-            BRA_CNT(2, 1);
-        }
-        record_error(status, BRA_ERR_TIMEOUT, t.b);
-        ok = false;
-        return false;
-    };
-    auto read_entries = [&](const TileCoord& t, int m) -> int2 {
-        if (FUSED && !wait_routed(t)) return make_int2(-1, -1);
-        return checked(index_entries(t, m));
     };
     auto load_k = [&](const TileCoord& t, int2 ent, int buf) {
         int r = lhead ? ent.y : ent.x;
@@ -413,393 +166,207 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
         }
     };
 
-    // ---- fused forward: pooling of one unit, and the routing of an image -------------------------------
-    // Pooling mirrors the stand-alone kernel for regions eight rows high: thread (row half yh, column tx,
-    // 16-byte channel vector c) sums its four token rows in order; then one thread per channel adds, column
-    // by column, (lower half + upper half).  The loader mapping above is exactly that thread grid.
-    auto pool_issue = [&](const Job& jb, uint4 (&pv)[8]) {
-        const size_t off = region_off(jb.pool_b, jb.i, jb.hp * 64);
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            pv[u] = ldg_nc_u4(Qb + off + u * row_bytes);
-            pv[4 + u] = ldg_nc_u4(Kb + off + u * row_bytes);
-        }
-    };
-    auto pool_finish = [&](const Job& jb, const uint4 (&pv)[8]) {
-        const uint32_t part = sm_base + OFF_POOL;        // [tensor][row half][column][64 ch] fp32
-#pragma unroll
-        for (int tsr = 0; tsr < 2; ++tsr) {
-            float acc[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint4 v = pv[4 * tsr + u];
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    acc[2 * e] += __uint_as_float(w[e] << 16);
-                    acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
-                }
-            }
-            const uint32_t dst = part + ((((tsr * 2 + head_half) * 8 + tx) * 64 + c * 8) << 2);
-            sts_f32x4(dst, acc[0], acc[1], acc[2], acc[3]);
-            sts_f32x4(dst + 16, acc[4], acc[5], acc[6], acc[7]);
-        }
-        __syncthreads();
-        {
-            const int tsr = tid >> 6, ch = tid & 63;
-            const uint32_t src = part + (((tsr * 2) * 8 * 64 + ch) << 2);
-            float s = 0.f;
-#pragma unroll
-            for (int x = 0; x < 8; ++x) s += lds_f32(src + x * 256) + lds_f32(src + 8 * 256 + x * 256);
-            float* dst = tsr ? fa.k_mean : fa.q_mean;
-            dst[((size_t)jb.pool_b * dm.R + jb.i) * dm.C + jb.hp * 64 + ch] = s * (1.0f / 64.0f);
-        }
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) {
-            const int done = atomicAdd(fa.pool_cnt + jb.pool_b, 1) + 1;
-            if (done == fa.units) __threadfence();
-            *last_slot = done == fa.units;
-        }
-        __syncthreads();
-#ifdef BRA_EXP_TRACE
-        long long tr0 = clock64();
-#endif
-        if (*last_slot) route_image(fa, dm, jb.pool_b, smem);
-#ifdef BRA_EXP_TRACE
-        if (*last_slot) { BRA_CNT(3, 1); BRA_CNT(4, (clock64() - tr0) >> 4); }
-#endif
-    };
-    auto decode_job = [&](int ticket) -> int4 {
-        int4 j = make_int4(-1, -1, 0, 0);
-        if (ticket < fa.total) {
-            const int s = ticket / fa.units, u = ticket - s * fa.units;
-            j.x = s >= fa.delta ? s - fa.delta : -1;
-            j.y = s < dm.B ? s : -1;
-            j.z = u / pairs;
-            j.w = u - j.z * pairs;
-        }
-        return j;
-    };
-
-    // ---- the jobs of this CTA ---------------------------------------------------------------------------
+    bool ok = true;
     uint32_t n_s = 0, n_o = 0;              // uses of bar_s / bar_o so far (phase parity)
-    TileWalker walk;
-    int tiles_left = 0;
-    Job cur, nxt;
-    if (FUSED) {
-        if (tid == 0) {
-            if (blockIdx.x == 0) { fa.ctrl[2] = fa.sync_off; fa.ctrl[3] = fa.sync_bytes; }
-            const int t0 = atomicAdd(fa.ctrl + 8, 1), t1 = atomicAdd(fa.ctrl + 8, 1);
-            job_slot[0] = decode_job(t0);
-            job_slot[1] = decode_job(t1);
-        }
-        __syncthreads();
-        const int4 a = job_slot[0], bq = job_slot[1];
-        cur = Job{a.x, a.y, a.z, a.w};
-        nxt = Job{bq.x, bq.y, bq.z, bq.w};
-        __syncthreads();
-    } else {
-        walk.init(blockIdx.x, gridDim.x, dm);
-        tiles_left = (num_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-        cur = Job{tiles_left > 0 ? walk.b : -1, -1, walk.i, walk.hp};
-        if (tiles_left > 1) { walk.next(); nxt = Job{walk.b, -1, walk.i, walk.hp}; }
-        else nxt = Job{-1, -1, 0, 0};
-    }
-    // copies of a tile go out in two groups: (Q, K of the first routed step), then (V, halo)
+    TileCoord t = coord_of(walk.b, walk.i, walk.hp);
+    // copies of a tile go out in two groups: (Q, K of the first routed step), then (V of that step, halo).
+    // Q and the V halo are inputs of the call: their copies (and everything above) overlap the tail of the
+    // kernel before (routing, in a forward call); only the routing index has to wait for it
+    if (my_tiles > 0) load_q(t);
+    pdl_wait();
     int2 ent = make_int2(0, 0);             // entries of the unit whose K/V are being loaded
-    auto issue_tile = [&](const TileCoord& t, bool have_entries) {
-        load_q(t);
-        if (!have_entries) ent = read_entries(t, 0);
+    if (my_tiles > 0) {
+        ent = read_entries(t, 0);
         load_k(t, ent, 0);
-        cp_async_commit();
-        load_v(t, ent, 0);
-        load_halo(t);
-        cp_async_commit();
-    };
-    if (cur.att_b >= 0) {
-        const TileCoord t = coord_of(cur.att_b, cur.i, cur.hp);
-        if (FUSED) {
-            issue_tile(t, false);
-        } else {
-            // Q and the V halo are inputs of the call: their copies (and everything above) overlap the tail
-            // of the kernel before (routing, in a forward call); only the routing index has to wait for it
-            load_q(t);
-            pdl_wait();
-            ent = read_entries(t, 0);
-            load_k(t, ent, 0);
-            cp_async_commit();
-            load_v(t, ent, 0);
-            load_halo(t);
-            cp_async_commit();
-        }
-    } else if (!FUSED) {
-        pdl_wait();
     }
+    cp_async_commit();
+    if (my_tiles > 0) { load_v(t, ent, 0); load_halo(t); }
+    cp_async_commit();
 
-    int n = 0;
-    while (cur.att_b >= 0 || cur.pool_b >= 0) {
-        int ticket2 = 0;
-        BRA_TR(n, 0);
-        BRA_TR(n, 9);
-        if (FUSED && tid == 0) ticket2 = atomicAdd(fa.ctrl + 8, 1);      // the job after next
-        uint4 pv[8];
-#ifdef BRA_EXP_POOL_EARLY
-        if (FUSED && cur.pool_b >= 0) pool_issue(cur, pv);
-#endif
-        const bool has_next = nxt.att_b >= 0;
-        const TileCoord tn = coord_of(has_next ? nxt.att_b : 0, nxt.i, nxt.hp);
+    for (int n = 0; n < my_tiles && ok; ++n) {
+        if (dm.lce && t.hp != hp_loaded) {
+            const float* wp = lce_w + (size_t)(t.c0 + 2 * lane) * 25;
+#pragma unroll
+            for (int q = 0; q < 25; ++q) wv[q] = make_float2(__ldg(wp + q), __ldg(wp + 25 + q));
+            if (lce_b) bias2 = make_float2(__ldg(lce_b + t.c0 + 2 * lane), __ldg(lce_b + t.c0 + 2 * lane + 1));
+            hp_loaded = t.hp;
+        }
+        const bool has_next = n + 1 < my_tiles;
+        if (has_next) walk.next();
+        const TileCoord tn = has_next ? coord_of(walk.b, walk.i, walk.hp) : t;
 
-        if (cur.att_b >= 0) {
-            const TileCoord t = coord_of(cur.att_b, cur.i, cur.hp);
-            if (!FUSED && dm.lce && t.hp != hp_loaded) {
-                const float* wp = lce_w + (size_t)(t.c0 + 2 * lane) * 25;
+        float m_run = -INFINITY, l_run = 0.f;
+        float o_acc[32];
 #pragma unroll
-                for (int q = 0; q < 25; ++q) wv_keep[q] = make_float2(__ldg(wp + q), __ldg(wp + 25 + q));
-                if (lce_b) bias_keep = make_float2(__ldg(lce_b + t.c0 + 2 * lane), __ldg(lce_b + t.c0 + 2 * lane + 1));
-                hp_loaded = t.hp;
-            }
-            float m_run = -INFINITY, l_run = 0.f;
-            bool next_routed = true;
-            float o_acc[32];
-#pragma unroll
-            for (int q = 0; q < 32; ++q) o_acc[q] = 0.f;
-            for (int m = 0; m < k; ++m) {
-                const int buf = K1 ? 0 : (m & 1);
-                const int2 ent_cur = ent;
-                // ---- Q and this step's K have landed; make them visible to the tensor core ----
-                if (m == 0) cp_async_wait<1>(); else cp_async_wait<0>();
-                fence_proxy_async_smem();
-                __syncthreads();
-                if (tid == 0) {
-                    tc_fence_after_sync();
-                    const uint32_t qa = sm_base + OFF_Q;
-                    const uint32_t ka = sm_base + (buf ? OFF_KV1 : OFF_K);
-#pragma unroll
-                    for (int ks = 0; ks < 2; ++ks)         // d = 32 = 2 k-steps of 16
-                        umma_ss(tmem, umma_smem_desc(qa + ks * 32, 16, 512, 4),
-                                umma_smem_desc(ka + ks * 32, 16, 512, 4), IDESC_S, ks);
-                    umma_commit(bar_s);
-                }
-                BRA_TR(n, 1);
-                // ---- fused forward: this job's pooling (and, once per image, its routing) while S is formed;
-                // before any wait on a flag, so that a wait only ever depends on jobs numbered below its own ----
-                if (FUSED && m == 0 && cur.pool_b >= 0) {
-#ifndef BRA_EXP_POOL_EARLY
-                    pool_issue(cur, pv);
-#endif
-                    pool_finish(cur, pv);
-                }
-                BRA_TR(n, 2);
-                // ---- next routed step of this tile: K/V into the other buffer (its MMAs are done) ----
-                const bool more = !K1 && m + 1 < k;
-                if (more) {
-                    ent = read_entries(t, m + 1);
-                    load_k(t, ent, buf ^ 1);
-                    load_v(t, ent, buf ^ 1);
-                    cp_async_commit();
-                } else if (has_next) {
-                    // in flight during the softmax.  Fused forward: a look only; the image may not be routed
-                    // yet, in which case the entries are read again after the last MMA of this tile
-                    if (FUSED) next_routed = ld_acquire_gpu(fa.route_flag + tn.b) != 0;
-                    ent = index_entries(tn, 0);
-                }
-                const bool valid = (head_half ? ent_cur.y : ent_cur.x) >= 0;
-                if (warp == 0) ok = mbar_wait(bar_s, n_s & 1, POLL_LIMIT) && ok;   // one warp polls, the rest sleep at the barrier
-                ++n_s;
-                if (!__syncthreads_and(ok)) { ok = false; break; }
-                tc_fence_after_sync();
-                BRA_TR(n, 3);
-                // pass 1: row maximum
-                float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll 1
-                for (int cc = 0; cc < 64; cc += 16) {
-                    uint32_t r[16];
-                    tmem_ld_32x32b_x16(s_addr + cc, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int q = 0; q < 16; q += 4) {
-                        m0 = fmax3(m0, __uint_as_float(r[q]), __uint_as_float(r[q + 1]));
-                        m1 = fmax3(m1, __uint_as_float(r[q + 2]), __uint_as_float(r[q + 3]));
-                    }
-                }
-                float mx = m_run;
-                if (valid) mx = fmaxf(mx, fmaxf(m0, m1) * sl2);               // sl2 > 0
-                const float corr = (mx == -INFINITY) ? 1.f : ex2f(m_run - mx);
-                const float mneg = (mx == -INFINITY) ? 0.f : -mx;
-                m_run = mx;
-                // pass 2: P = exp2(S * scale * log2 e - max), bf16 pairs written over the columns
-                // of S already consumed (column j of P never outruns column 2j of S); row sum
-                const float2 sl2v = make_float2(sl2, sl2), mnegv = make_float2(mneg, mneg);
-                float2 sum2 = make_float2(0.f, 0.f);
-#pragma unroll 1
-                for (int cc = 0; cc < 64; cc += 16) {
-                    uint32_t r[16], pk[8];
-                    tmem_ld_32x32b_x16(s_addr + cc, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int q = 0; q < 16; q += 2) {
-                        const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[q]), __uint_as_float(r[q + 1])), sl2v, mnegv);
-                        const float2 pe = make_float2(valid ? ex2f(a.x) : 0.f, valid ? ex2f(a.y) : 0.f);
-                        sum2 = __fadd2_rn(sum2, pe);
-                        pk[q >> 1] = pack_bf16(pe.x, pe.y);
-                    }
-                    tmem_st_32x32b_x8(p_addr + (cc >> 1), pk);
-                }
-                tmem_st_wait();
-                // this step's V has landed (first step: the group of V and the halo, which leaves the copies
-                // of the next routed step, if any, in flight)
-                if (m == 0) {
-                    if (more) cp_async_wait<1>(); else cp_async_wait<0>();
-                    fence_proxy_async_smem();
-                }
-                tc_fence_before_sync();
-                __syncthreads();
-                BRA_TR(n, 4);
-                if (tid == 0) {
-                    tc_fence_after_sync();
-                    const uint64_t vd = umma_smem_desc(sm_base + (buf ? OFF_KV1 + 8192 : OFF_V), 16, 1024, 2);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)         // 64 keys = 4 k-steps of 16 (2048 B of V each)
-                        umma_ts(tmem + TM_O, tmem + ks * 8, vd + (uint64_t)(ks * 128), IDESC_O, ks);
-                    umma_commit(bar_o);
-                }
-                if (warp == 0) ok = mbar_wait(bar_o, n_o & 1, POLL_LIMIT) && ok;
-                ++n_o;
-                if (!__syncthreads_and(ok)) { ok = false; break; }
-                tc_fence_after_sync();
-                BRA_TR(n, 5);
-                uint32_t oraw[32];
-                tmem_ld_32x32b_x32(o_addr, oraw);
-                tmem_ld_wait();
-                tc_fence_before_sync();
-                if (K1) {
-                    l_run = sum2.x + sum2.y;
-#pragma unroll
-                    for (int q = 0; q < 32; ++q) o_acc[q] = __uint_as_float(oraw[q]);
-                } else {
-                    l_run = fmaf(l_run, corr, sum2.x + sum2.y);
-#pragma unroll
-                    for (int q = 0; q < 32; ++q) o_acc[q] = fmaf(o_acc[q], corr, __uint_as_float(oraw[q]));
-                }
-            }
-            if (!ok) break;
-
-            // every MMA of this tile has read its operands: Q and K (buffer 0) of the next tile go out now
-            if (has_next) {
-                load_q(tn);
-                if (FUSED && !next_routed) { BRA_CNT(0, 1); ent = wait_routed(tn) ? index_entries(tn, 0) : make_int2(-1, -1); }
-                BRA_CNT(1, 1);
-                ent = checked(ent);
-                load_k(tn, ent, 0);
-            }
-            cp_async_commit();
-            // ---- normalise, stage O^att as fp32 [64 tokens][64 ch] (16-byte units xor-swizzled) ----
-            {
-                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                const uint32_t srow = sm_base + OFF_ST + tq * 256;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const int chunk = head_half * 8 + q;
-                    sts_f32x4(srow + ((chunk ^ (tq & 7)) << 4),
-                              o_acc[4 * q] * inv, o_acc[4 * q + 1] * inv, o_acc[4 * q + 2] * inv, o_acc[4 * q + 3] * inv);
-                }
-                if (lse)
-                    lse[((size_t)t.b * dm.heads + 2 * t.hp + head_half) * dm.N + (size_t)(t.y0 + tq / RS) * dm.W + t.x0 + tq % RS] =
-                        (m_run + log2f(l_run)) * 0.6931471805599453f;
-            }
+        for (int q = 0; q < 32; ++q) o_acc[q] = 0.f;
+        for (int m = 0; m < k; ++m) {
+            const int buf = m & 1;
+            const int2 ent_cur = ent;
+            // ---- Q and this step's K have landed; make them visible to the tensor core ----
+            if (m == 0) cp_async_wait<1>(); else cp_async_wait<0>();
+            fence_proxy_async_smem();
             __syncthreads();
-            BRA_TR(n, 6);
-
-            // ---- LCE + store ----
-            // Input row yy of the halo feeds output rows yy - ti through tap row ti.  Fully unrolled:
-            // the 8 x 2 output sums of this thread's channel pair sit in registers under fixed names,
-            // starting from O^att (+ bias).
-            {
-                const uint32_t halo = sm_base + OFF_HALO + (xl0 * 32 + lane) * 4;
-                const uint32_t stage = sm_base + OFF_ST + xl0 * 256 + (lane & 1) * 8;
-                uint32_t* out = reinterpret_cast<uint32_t*>(O) +
-                                ((((size_t)t.b * dm.H + t.y0) * dm.W + t.x0 + xl0) * dm.C + t.c0) / 2 + lane;
-                const size_t out_row = (size_t)dm.W * (dm.C / 2);
-                // staging token tk = y * 8 + xl0 + xx: its 16-byte unit index is xor-ed with tk & 7
-                const uint32_t sw0 = (((lane >> 1) ^ (xl0 & 7)) << 4), sw1 = (((lane >> 1) ^ ((xl0 + 1) & 7)) << 4);
-                float2 wv[25];
-                float2 bias2 = bias_keep;
-                if (FUSED) {
-                    if (dm.lce) {
-                        const float* wp = lce_w + (size_t)(t.c0 + 2 * lane) * 25;
+            if (tid == 0) {
+                tc_fence_after_sync();
+                const uint32_t qa = sm_base + OFF_Q;
+                const uint32_t ka = sm_base + (buf ? OFF_KV1 : OFF_K);
 #pragma unroll
-                        for (int q = 0; q < 25; ++q) wv[q] = make_float2(__ldg(wp + q), __ldg(wp + 25 + q));
-                        if (lce_b) bias2 = make_float2(__ldg(lce_b + t.c0 + 2 * lane), __ldg(lce_b + t.c0 + 2 * lane + 1));
-                    }
-                } else {
+                for (int ks = 0; ks < 2; ++ks)         // d = 32 = 2 k-steps of 16
+                    umma_ss(tmem, umma_smem_desc(qa + ks * 32, 16, 512, 4),
+                            umma_smem_desc(ka + ks * 32, 16, 512, 4), IDESC_S, ks);
+                umma_commit(bar_s);
+            }
+            // ---- next routed step of this tile: K/V into the other buffer (its MMAs are done) ----
+            const bool more = m + 1 < k;
+            if (more) {
+                ent = read_entries(t, m + 1);
+                load_k(t, ent, buf ^ 1);
+                load_v(t, ent, buf ^ 1);
+                cp_async_commit();
+            } else if (has_next) {
+                ent = read_entries(tn, 0);             // in flight during the softmax
+            }
+            const bool valid = (head_half ? ent_cur.y : ent_cur.x) >= 0;
+            if (warp == 0) ok = mbar_wait(bar_s, n_s & 1, POLL_LIMIT);   // one warp polls, the rest sleep at the barrier
+            ++n_s;
+            if (!__syncthreads_and(ok)) { ok = false; break; }
+            tc_fence_after_sync();
+            // pass 1: row maximum
+            float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll 1
+            for (int cc = 0; cc < 64; cc += 16) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(s_addr + cc, r);
+                tmem_ld_wait();
 #pragma unroll
-                    for (int q = 0; q < 25; ++q) wv[q] = wv_keep[q];
-                }
-                float2 acc[8][2];
-#pragma unroll
-                for (int y = 0; y < 8; ++y)
-#pragma unroll
-                    for (int xx = 0; xx < 2; ++xx)
-                        acc[y][xx] = __fadd2_rn(lds_f32x2(stage + (y * RS + xx) * 256 + (xx ? sw1 : sw0)), bias2);
-                if (dm.lce) {
-#pragma unroll
-                    for (int yy = 0; yy < HALO; ++yy) {
-                        float2 v[6];
-#pragma unroll
-                        for (int xx = 0; xx < 6; ++xx) {
-                            const uint32_t w = lds_u32(halo + (yy * HALO + xx) * 128);
-                            v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-                        }
-                        // tap column outermost: consecutive FMAs go to different sums
-#pragma unroll
-                        for (int tj = 0; tj < 5; ++tj)
-#pragma unroll
-                            for (int ti = 0; ti < 5; ++ti) {
-                                const int y = yy - ti;
-                                if (y < 0 || y >= 8) continue;
-#pragma unroll
-                                for (int xx = 0; xx < 2; ++xx)
-                                    acc[y][xx] = __ffma2_rn(wv[ti * 5 + tj], v[xx + tj], acc[y][xx]);
-                            }
-                    }
-                }
-#pragma unroll
-                for (int y = 0; y < 8; ++y) {
-#pragma unroll
-                    for (int xx = 0; xx < 2; ++xx) out[xx * (dm.C / 2)] = pack_bf16(acc[y][xx].x, acc[y][xx].y);
-                    out += out_row;
+                for (int q = 0; q < 16; q += 4) {
+                    m0 = fmax3(m0, __uint_as_float(r[q]), __uint_as_float(r[q + 1]));
+                    m1 = fmax3(m1, __uint_as_float(r[q + 2]), __uint_as_float(r[q + 3]));
                 }
             }
-        } else {
-            // a job without an attention part (the first delta image slots): pooling only
-#ifndef BRA_EXP_POOL_EARLY
-            pool_issue(cur, pv);
-#endif
-            pool_finish(cur, pv);
+            float mx = m_run;
+            if (valid) mx = fmaxf(mx, fmaxf(m0, m1) * sl2);               // sl2 > 0
+            const float corr = (mx == -INFINITY) ? 1.f : ex2f(m_run - mx);
+            const float mneg = (mx == -INFINITY) ? 0.f : -mx;
+            m_run = mx;
+            // pass 2: P = exp2(S * scale * log2 e - max), bf16 pairs written over the columns
+            // of S already consumed (column j of P never outruns column 2j of S); row sum
+            const float2 sl2v = make_float2(sl2, sl2), mnegv = make_float2(mneg, mneg);
+            float2 sum2 = make_float2(0.f, 0.f);
+#pragma unroll 1
+            for (int cc = 0; cc < 64; cc += 16) {
+                uint32_t r[16], pk[8];
+                tmem_ld_32x32b_x16(s_addr + cc, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 16; q += 2) {
+                    const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[q]), __uint_as_float(r[q + 1])), sl2v, mnegv);
+                    const float2 pe = make_float2(valid ? ex2f(a.x) : 0.f, valid ? ex2f(a.y) : 0.f);
+                    sum2 = __fadd2_rn(sum2, pe);
+                    pk[q >> 1] = pack_bf16(pe.x, pe.y);
+                }
+                tmem_st_32x32b_x8(p_addr + (cc >> 1), pk);
+            }
+            tmem_st_wait();
+            // first step: the group of V and the halo has landed (the copies of the next routed step stay in flight)
+            if (m == 0) {
+                if (more) cp_async_wait<1>(); else cp_async_wait<0>();
+                fence_proxy_async_smem();
+            }
+            tc_fence_before_sync();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after_sync();
+                const uint64_t vd = umma_smem_desc(sm_base + (buf ? OFF_KV1 + 8192 : OFF_V), 16, 1024, 2);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)         // 64 keys = 4 k-steps of 16 (2048 B of V each)
+                    umma_ts(tmem + TM_O, tmem + ks * 8, vd + (uint64_t)(ks * 128), IDESC_O, ks);
+                umma_commit(bar_o);
+            }
+            if (warp == 0) ok = mbar_wait(bar_o, n_o & 1, POLL_LIMIT);
+            ++n_o;
+            if (!__syncthreads_and(ok)) { ok = false; break; }
+            tc_fence_after_sync();
+            uint32_t oraw[32];
+            tmem_ld_32x32b_x32(o_addr, oraw);
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            l_run = fmaf(l_run, corr, sum2.x + sum2.y);
+#pragma unroll
+            for (int q = 0; q < 32; ++q) o_acc[q] = fmaf(o_acc[q], corr, __uint_as_float(oraw[q]));
         }
-        BRA_TR(n, 7);
-        if (FUSED && tid == 0) job_slot[n & 1] = decode_job(ticket2);
-        __syncthreads();                    // staging tile (over V) and halo are free
-        BRA_TR(n, 8);
-        if (cur.att_b >= 0) {
-            if (has_next) { load_v(tn, ent, 0); load_halo(tn); }
-            cp_async_commit();
-        } else {
-            if (has_next) issue_tile(tn, false); else { cp_async_commit(); }
+        if (!ok) break;
+
+        // every MMA of this tile has read its operands: Q and K (buffer 0) of the next tile go out now
+        if (has_next) { load_q(tn); load_k(tn, ent, 0); }
+        cp_async_commit();
+        // ---- normalise, stage O^att as fp32 [64 tokens][64 ch] (16-byte units xor-swizzled) ----
+        {
+            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            const uint32_t srow = sm_base + OFF_ST + tq * 256;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int chunk = head_half * 8 + q;
+                sts_f32x4(srow + ((chunk ^ (tq & 7)) << 4),
+                          o_acc[4 * q] * inv, o_acc[4 * q + 1] * inv, o_acc[4 * q + 2] * inv, o_acc[4 * q + 3] * inv);
+            }
+            if (lse)
+                lse[((size_t)t.b * dm.heads + 2 * t.hp + head_half) * dm.N + (size_t)(t.y0 + tq / RS) * dm.W + t.x0 + tq % RS] =
+                    (m_run + log2f(l_run)) * 0.6931471805599453f;
         }
-        cur = nxt;
-        if (FUSED) {
-            const int4 a = job_slot[n & 1];
-            nxt = Job{a.x, a.y, a.z, a.w};
-        } else {
-            --tiles_left;
-            if (tiles_left > 1) { walk.next(); nxt = Job{walk.b, -1, walk.i, walk.hp}; }
-            else nxt = Job{-1, -1, 0, 0};
+        __syncthreads();
+
+        // ---- LCE + store ----
+        // Input row yy of the halo feeds output rows yy - ti through tap row ti.  Fully unrolled:
+        // the 8 x 2 output sums of this thread's channel pair sit in registers under fixed names,
+        // starting from O^att (+ bias).
+        {
+            const uint32_t halo = sm_base + OFF_HALO + (xl0 * 32 + lane) * 4;
+            const uint32_t stage = sm_base + OFF_ST + xl0 * 256 + (lane & 1) * 8;
+            uint32_t* out = reinterpret_cast<uint32_t*>(O) +
+                            ((((size_t)t.b * dm.H + t.y0) * dm.W + t.x0 + xl0) * dm.C + t.c0) / 2 + lane;
+            const size_t out_row = (size_t)dm.W * (dm.C / 2);
+            // staging token tk = y * 8 + xl0 + xx: its 16-byte unit index is xor-ed with tk & 7
+            const uint32_t sw0 = (((lane >> 1) ^ (xl0 & 7)) << 4), sw1 = (((lane >> 1) ^ ((xl0 + 1) & 7)) << 4);
+            float2 acc[8][2];
+#pragma unroll
+            for (int y = 0; y < 8; ++y)
+#pragma unroll
+                for (int xx = 0; xx < 2; ++xx)
+                    acc[y][xx] = __fadd2_rn(lds_f32x2(stage + (y * RS + xx) * 256 + (xx ? sw1 : sw0)), bias2);
+            if (dm.lce) {
+#pragma unroll
+                for (int yy = 0; yy < HALO; ++yy) {
+                    float2 v[6];
+#pragma unroll
+                    for (int xx = 0; xx < 6; ++xx) {
+                        const uint32_t w = lds_u32(halo + (yy * HALO + xx) * 128);
+                        v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+                    }
+                    // tap column outermost: consecutive FMAs go to different sums
+#pragma unroll
+                    for (int tj = 0; tj < 5; ++tj)
+#pragma unroll
+                        for (int ti = 0; ti < 5; ++ti) {
+                            const int y = yy - ti;
+                            if (y < 0 || y >= 8) continue;
+#pragma unroll
+                            for (int xx = 0; xx < 2; ++xx)
+                                acc[y][xx] = __ffma2_rn(wv[ti * 5 + tj], v[xx + tj], acc[y][xx]);
+                        }
+                }
+            }
+#pragma unroll
+            for (int y = 0; y < 8; ++y) {
+#pragma unroll
+                for (int xx = 0; xx < 2; ++xx) out[xx * (dm.C / 2)] = pack_bf16(acc[y][xx].x, acc[y][xx].y);
+                out += out_row;
+            }
         }
-        ++n;
+        __syncthreads();                    // staging tile (over V, buffer 0) and halo are free
+        if (has_next) { load_v(tn, ent, 0); load_halo(tn); }
+        cp_async_commit();
+        t = tn;
     }
 
     // ---- teardown: nothing in flight, TMEM returned ----
@@ -812,116 +379,36 @@ attend_tc_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __re
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (FUSED) {
-        // the last CTA to finish puts the counters and flags back to zero for the next call
-        if (tid == 0) {
-            __threadfence();
-            *last_slot = atomicAdd(fa.ctrl + 9, 1) == (int)gridDim.x - 1;
-        }
-        __syncthreads();
-        if (*last_slot && ok) {
-            for (int e = tid; e < dm.B; e += THREADS) { fa.pool_cnt[e] = 0; fa.route_flag[e] = 0; }
-            if (tid == 0) { fa.ctrl[8] = 0; fa.ctrl[9] = 0; }
-        }
-    }
 }
 
 // ------------------------------------------------------------------ host side
-static int sm_count() {
-    static int n[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
-    if (!n[dev] && cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n[dev] = 1;
-    return n[dev] > 0 ? n[dev] : 1;
-}
-
 bool attend_tc_supported(const Dims& d, int dtype) {
     return dtype == BRA_BF16 && d.d == 32 && d.heads % 2 == 0 && d.hs == tc::RS && d.ws == tc::RS &&
            d.topk <= tc::KCAP && (long long)d.B * d.R * (d.heads / 2) < (1ll << 30) &&
            (long long)d.W * d.C * 2 * tc::HALO < (1ll << 31) && d.R <= 4096;
 }
 
-// The one-launch forward: per-head routing with k = 1, at most 64 regions, and a channel count for which
-// the stand-alone pooling kernel sums in the same order (so that bra_forward and bra_route agree bit for bit).
-bool forward_tc_supported(const Dims& d, int dtype) {
-    return attend_tc_supported(d, dtype) && d.topk == 1 && d.heads_i == d.heads && d.R <= tc::FUSED_MAX_R &&
-           d.C <= 128 && ((long long)d.B + 64) * d.R * (d.heads / 2) < (1ll << 30);
-}
-
-static cudaError_t set_attributes() {
-    static PerDeviceOnce once;
-    return once.run([]() -> cudaError_t {
-        cudaError_t e;
-        if ((e = cudaFuncSetAttribute(attend_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_K1)) != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(attend_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_K1)) != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(attend_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_KN)) != cudaSuccess) return e;
-        // several CTAs per SM: ask for the largest shared-memory carve-out
-        if ((e = cudaFuncSetAttribute(attend_tc_kernel<true, false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(attend_tc_kernel<true, true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
-        return cudaFuncSetAttribute(attend_tc_kernel<false, false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    });
-}
-
 cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const void* V,
                              const int32_t* index, const float* lce_w, const float* lce_b,
                              void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel) {
-    cudaError_t e = set_attributes();
+    if (d.topk == 1) return launch_attend_tc_k1(d, Q, K, V, index, lce_w, lce_b, O, lse, status, st, after_own_kernel);
+    static PerDeviceOnce once;
+    cudaError_t e = once.run([]() -> cudaError_t {
+        cudaError_t a = cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_KN);
+        if (a != cudaSuccess) return a;
+        // several CTAs per SM: ask for the largest shared-memory carve-out
+        return cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    });
     if (e != cudaSuccess) return e;
     const int tiles = d.B * d.R * (d.heads / 2);
-    const int resident = sm_count() * (d.topk == 1 ? 4 : 3);
+    const int resident = tc_sm_count() * 3;
     const unsigned grid = (unsigned)(tiles < resident ? tiles : resident);
-    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(Q);
-    const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(K);
-    const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(V);
-    __nv_bfloat16* o = static_cast<__nv_bfloat16*>(O);
-    const FusedArgs none = {};
-    if (d.topk == 1)
-        e = launch_kernel(attend_tc_kernel<true, false>, dim3(grid), dim3(tc::THREADS), tc::SMEM_K1, st, after_own_kernel,
-                          q, k, v, index, lce_w, lce_b, o, lse, status, d, tiles, none);
-    else
-        e = launch_kernel(attend_tc_kernel<false, false>, dim3(grid), dim3(tc::THREADS), tc::SMEM_KN, st, after_own_kernel,
-                          q, k, v, index, lce_w, lce_b, o, lse, status, d, tiles, none);
-    count_launch();
-    return e;
-}
-
-cudaError_t launch_forward_tc(const Dims& d, const void* Q, const void* K, const void* V,
-                              const float* lce_w, const float* lce_b, void* O, int32_t* index, float* lse,
-                              float* q_mean, float* k_mean, int32_t* ctrl, int32_t* sync, int inject,
-                              cudaStream_t st) {
-    cudaError_t e = set_attributes();
-    if (e != cudaSuccess) return e;
-    FusedArgs fa;
-    fa.q_mean = q_mean; fa.k_mean = k_mean; fa.index_out = index;
-    fa.pool_cnt = sync; fa.route_flag = sync + d.B; fa.ctrl = ctrl;
-    fa.units = d.R * (d.heads / 2);
-    const int resident = sm_count() * 4;
-    // pooling runs this many images ahead of attention: the jobs of one wave of resident CTAs, plus the
-    // time the routing of an image takes after its last unit is pooled
-    int delta = (resident + fa.units - 1) / fa.units + 3;
-    static const char* env = getenv("BRA_FUSED_DELTA");               // tuning aid
-    if (env && atoi(env) > 0) delta = atoi(env);
-    fa.delta = delta < d.B ? delta : d.B;
-    fa.total = (d.B + fa.delta) * fa.units;
-    fa.inject = inject;
-    fa.sync_off = (int)(reinterpret_cast<char*>(sync) - reinterpret_cast<char*>(ctrl));
-    fa.sync_bytes = (int)(sizeof(int32_t) * 2 * (size_t)d.B);
-    const unsigned grid = (unsigned)(fa.total < resident ? fa.total : resident);
-    e = launch_kernel(attend_tc_kernel<true, true>, dim3(grid), dim3(tc::THREADS), tc::SMEM_K1, st, false,
+    e = launch_kernel(attend_tc_kernel, dim3(grid), dim3(tc::THREADS), tc::SMEM_KN, st, after_own_kernel,
                       static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
-                      static_cast<const __nv_bfloat16*>(V), static_cast<const int32_t*>(index), lce_w, lce_b,
-                      static_cast<__nv_bfloat16*>(O), lse, ctrl, d, 0, fa);
+                      static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b,
+                      static_cast<__nv_bfloat16*>(O), lse, status, d, tiles);
     count_launch();
     return e;
 }
 
 }  // namespace bra
-
-#ifdef BRA_EXP_TRACE
-extern "C" int bra_debug_read_trace(long long* out, int* cnt) {
-    cudaMemcpyFromSymbol(out, bra::g_trace, sizeof(bra::g_trace));
-    cudaMemcpyFromSymbol(cnt, bra::g_trace_cnt, sizeof(bra::g_trace_cnt));
-    int z[16] = {};
-    return (int)cudaMemcpyToSymbol(bra::g_trace_cnt, z, sizeof(z));
-}
-#endif

@@ -40,7 +40,7 @@ static bra_status make_dims(const bra_problem* p, Dims* out) {
     if (p->topk < 1 || (int64_t)p->topk > (int64_t)p->S * p->S) return BRA_ERR_TOPK;
     if (p->dtype != BRA_F32 && p->dtype != BRA_BF16) return BRA_ERR_DTYPE;
     if (p->lce_ksize != 0 && p->lce_ksize != 5) return BRA_ERR_UNSUPPORTED;
-    if (p->impl < BRA_IMPL_AUTO || p->impl > BRA_IMPL_IMG) return BRA_ERR_UNSUPPORTED;
+    if (p->impl < BRA_IMPL_AUTO || p->impl > BRA_IMPL_TC_FUSED) return BRA_ERR_UNSUPPORTED;
     if (p->inject != BRA_INJECT_NONE && p->inject != BRA_INJECT_HOLD_ROUTE_FLAGS) return BRA_ERR_UNSUPPORTED;
     Dims d;
     d.B = p->B; d.H = p->H; d.W = p->W; d.C = p->C; d.heads = p->heads; d.S = p->S; d.topk = p->topk;
@@ -79,6 +79,7 @@ static Path choose_attend(const Dims& d, int dtype, int impl) {
     switch (impl) {
         case BRA_IMPL_SIMT: return attend_simt_supported(d) ? PATH_SIMT : PATH_NONE;
         case BRA_IMPL_MMA:  return attend_mma_supported(d, dtype) ? PATH_MMA : PATH_NONE;
+        case BRA_IMPL_TC_FUSED: return attend_tc_supported(d, dtype) ? PATH_TC : PATH_NONE;
         case BRA_IMPL_TC:   return attend_tc_supported(d, dtype) ? PATH_TC
                                  : attend_tc_wide_supported(d, dtype) ? PATH_TC_WIDE : PATH_NONE;
         case BRA_IMPL_IMG:  return attend_img_supported(d, dtype) ? PATH_IMG : PATH_NONE;
@@ -191,9 +192,9 @@ bra_status bra_forward(const bra_problem* p, const void* Q, const void* K, const
     int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
     float* qm = reinterpret_cast<float*>(w + L.q_mean);
     float* km = reinterpret_cast<float*>(w + L.k_mean);
-    // pooling, routing and attention in one launch where the tcgen05 kernel can do all three
-    static const bool no_fused = getenv("BRA_NO_FUSED") != nullptr;    // debugging aid: the three-launch chain
-    if (path == PATH_TC && !no_fused && forward_tc_supported(d, p->dtype)) {
+    // pooling, routing and attention in one launch, on request
+    if (p->impl == BRA_IMPL_TC_FUSED) {
+        if (!forward_tc_supported(d, p->dtype)) return BRA_ERR_UNSUPPORTED;
         const cudaError_t e = launch_forward_tc(d, Q, K, V, lce_w, lce_b, O, idx, lse, qm, km, status,
                                                 reinterpret_cast<int32_t*>(w + L.sync), p->inject, st);
         return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;

@@ -438,8 +438,9 @@ def test_forward_orders_attention_after_routing(bra, n):
         assert (idx == idx_ref).all() and (O == O_ref).all(), f"call {it}"
 
 
-# bf16, head dim 32, 8 x 8-token regions, topk = 1, per-head routing, <= 64 regions, C <= 128:
-# bra_forward is ONE kernel launch (pooling, routing and attention as numbered jobs of one grid)
+# bf16, head dim 32, 8 x 8-token regions, topk = 1, per-head routing, <= 64 regions, C <= 128: with
+# BRA_IMPL_TC_FUSED bra_forward is ONE kernel launch (pooling, routing and attention as numbered jobs of one grid)
+FUSED = 5
 ONE_LAUNCH_CASES = [
     BraConfig("fused-single-region", 1, 8, 8, 64, 2, 1, 1, "bf16"),
     BraConfig("fused-one-image", 1, 56, 56, 64, 2, 7, 1, "bf16"),
@@ -456,7 +457,7 @@ def test_forward_in_one_launch_equals_route_then_attend(bra, cfg):
     call after call on the same scratch buffer (its counters and flags clean themselves), and matches
     the oracle."""
     import torch
-    p = problem_of(bra, cfg)
+    p = problem_of(bra, cfg, impl=FUSED)
     ws = bra.workspace(p)
     sets = [to_dev(synthetic.make_inputs(cfg, seed=300 + s, clustered=bool(s)), cfg) for s in range(2)]
     want = []
@@ -485,11 +486,11 @@ def test_bounded_wait_that_runs_out_is_reported_and_recoverable(bra):
     reads BRA_ERR_TIMEOUT.  Reading the status restores the scratch buffer: the next call is clean."""
     cfg = BraConfig("timeout", 3, 32, 32, 64, 2, 4, 1, "bf16")
     t = to_dev(synthetic.make_inputs(cfg, seed=9), cfg)
-    p = problem_of(bra, cfg)
+    p = problem_of(bra, cfg, impl=FUSED)
     ws = bra.workspace(p)
     O_ref, idx_ref, _ = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
     assert bra.bra_device_status(ws) == 0
-    p_bad = problem_of(bra, cfg, inject=1)
+    p_bad = problem_of(bra, cfg, impl=FUSED, inject=1)
     bra.bra_forward(p_bad, t["Q"], t["K"], t["V"], t["w"], ws=ws)
     assert bra.bra_device_status(ws) == 10
     assert bra.bra_device_status(ws) == 0          # cleared by the read
@@ -505,7 +506,7 @@ def test_workspace_init_makes_a_dirty_buffer_usable(bra):
     import torch
     cfg = BraConfig("dirty-ws", 2, 32, 32, 64, 2, 4, 1, "bf16")
     t = to_dev(synthetic.make_inputs(cfg, seed=10), cfg)
-    p = problem_of(bra, cfg)
+    p = problem_of(bra, cfg, impl=FUSED)
     O_ref, idx_ref, _ = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"])
     ws = bra.workspace(p)
     ws.fill_(0xFF)
