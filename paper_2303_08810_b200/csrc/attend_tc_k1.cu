@@ -2,35 +2,51 @@
 // (Eq. 6, Eq. 7 with Eq. 1): every query region attends to one routed region per head, so a tile
 // needs one S = Q K^T, one softmax without running maximum, and one O = P V.
 //
-// Tile layout, thread mappings and shared-memory map are those of attend_tc.cu (two heads stacked
-// into a 128-row MMA tile, 128-thread CTAs, four per SM).  What differs is the schedule: the tensor
-// core works one tile ahead of the threads.  While the threads run the softmax and P V of tile n,
-// Q and K of tile n + 1 stream into the buffers S_n has just released; S_{n+1} = Q K^T is issued
-// before the LCE of tile n starts and completes underneath it, so a tile never waits for its first
-// MMA.  V of tile n + 1 follows once the staging tile that overlays it has been read, the halo
-// once the LCE is done.  Per tile:
-//   wait S_n (issued during tile n - 1)  ->  copies of Q, K of tile n + 1 go out
-//   softmax, P to TMEM  ->  O = P V  ->  normalised O^att to the fp32 staging tile
-//   S_{n+1} issued  ->  LCE sums start from O^att  ->  copy of V of tile n + 1 goes out
-//   LCE (5x5 depthwise correlation of V from the halo tile), one bf16 store of O
-//   ->  copy of the halo of tile n + 1 goes out
-// Every wait on an MMA is bounded.
+// Tile layout and thread mappings are those of attend_tc.cu (two heads stacked into a 128-row MMA
+// tile, 128-thread CTAs, four per SM).  Two things differ.
+//
+// Copies: the tiles reach shared memory as bulk tensor copies (TMA) issued by one thread: per tile
+// two {32 ch, 8, 8} boxes each of Q, of K and of V (one per head; the gather of Eq. 6 is the box
+// coordinates of the routed regions) in the 64-byte swizzled layout the MMA descriptors name, and
+// one {64 ch, 12, 12} box of V around the query region for the LCE, zero-filled outside the map (the
+// conv's padding).  Measured on B200 with four CTAs per SM these boxes fill shared memory at
+// 10-11 TB/s against 8.5 TB/s for per-thread 16-byte copies, and cost the other 127 threads no
+// address arithmetic at all.  Tensor maps cover this GPU's own memory; nothing is multicast.
+//
+// Schedule: the tensor core works one tile ahead of the threads.  While the threads run the softmax
+// and P V of tile n, Q and K of tile n + 1 land in the buffers S_n has released; S_{n+1} = Q K^T is
+// issued before the LCE of tile n starts and completes underneath it.  V of tile n + 1 follows once
+// the staging tile that overlays it has been read, the halo once the LCE is done.  Per tile:
+//   wait S_n  ->  copies of Q, K of tile n + 1 go out  ->  softmax, P to TMEM  ->  O = P V (two
+//   MMAs, one per head's V tile)  ->  normalised O^att to the fp32 staging tile  ->  S_{n+1} issued
+//   ->  LCE sums start from O^att  ->  copy of V of tile n + 1 goes out  ->  LCE (5x5 depthwise
+//   correlation of V from the halo tile), one bf16 store of O  ->  copy of the halo of tile n + 1.
+// Every wait (on an MMA, on a copy) is bounded.
 #include "attend_tc_common.cuh"
 
 namespace bra {
 
+namespace k1 {
+constexpr int OFF_VB = tc::OFF_V + 4096;        // head B's V tile ([64 keys][64 B], 64-byte swizzle), after head A's
+constexpr uint32_t QK_BYTES = 16384, V_BYTES = 8192;
+}  // namespace k1
+
+struct K1Maps { CUtensorMap q, k, v, halo; };   // {32 ch, 8, 8} boxes of Q, K, V; {64 ch, 12, 12} box of V
+
 __global__ void __launch_bounds__(tc::THREADS, 4)
-attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
-                 const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
-                 const float* __restrict__ lce_w, const float* __restrict__ lce_b,
-                 __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
-                 int32_t* __restrict__ status, Dims dm, int num_tiles) {
+attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
+                    const float* __restrict__ lce_w, const float* __restrict__ lce_b,
+                    __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
+                    int32_t* __restrict__ status, Dims dm, int num_tiles) {
     using namespace tc;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem + OFF_BAR);       // S landed in TMEM
     uint64_t* bar_o = bar_s + 1;                                         // O landed in TMEM
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_s + 2);
+    uint64_t* bar_qk = bar_s + 2;                                        // Q and K tiles landed in shared memory
+    uint64_t* bar_v = bar_s + 3;                                         // V tiles landed
+    uint64_t* bar_h = bar_s + 4;                                         // halo landed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_s + 5);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int inv_s = (1 << 20) / dm.S + 1;            // i / S == (i * inv_s) >> 20 for i < 4096
@@ -39,6 +55,9 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
     if (tid == 0) {
         mbar_init(bar_s, 1);
         mbar_init(bar_o, 1);
+        mbar_init(bar_qk, 1);
+        mbar_init(bar_v, 1);
+        mbar_init(bar_h, 1);
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(tmem_slot, TMEM_COLS);
@@ -48,23 +67,7 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
     const uint32_t tmem = *tmem_slot;
     TileWalker walk;
     walk.init(blockIdx.x, gridDim.x, dm);
-
-    // ---- loader mapping: thread copies 16-byte chunk c of the 128-byte channel row (both
-    // heads) of token column tx, in token rows lrow..lrow+3 of a region: a warp covers 512
-    // contiguous bytes per instruction.  Chunks 0-3 are head A, 4-7 head B; inside a head's
-    // [token][64 B] tile the chunk index is xor-ed with (token >> 1) & 3 (64-byte swizzle).
-    const int c = tid & 7, tx = (tid >> 3) & 7, lrow = (tid >> 6) * 4;
-    const int lhead = c >> 2;
-    const uint32_t tile_off = lhead * 4096 + (lrow * 8 + tx) * 64 + (((c & 3) ^ ((tx >> 1) & 3)) << 4);
-    // V: [key][128 B] with both heads side by side, 16-byte chunk index xor-ed with key & 7 (= tx)
-    const uint32_t v_off = (lrow * 8 + tx) * 128 + ((c ^ tx) << 4);
-    const size_t row_bytes = (size_t)dm.W * dm.C * 2;
-    const size_t img_bytes = (size_t)dm.H * row_bytes;
-    const size_t thr_off = (size_t)lrow * row_bytes + (size_t)tx * dm.C * 2 + c * 16;   // this thread's chunk inside a region
     const uint32_t sm_base = smem_u32(smem);
-    const uint8_t* Qb = reinterpret_cast<const uint8_t*>(Qg);
-    const uint8_t* Kb = reinterpret_cast<const uint8_t*>(Kg);
-    const uint8_t* Vb = reinterpret_cast<const uint8_t*>(Vg);
 
     // ---- softmax mapping: thread = row of the stacked tile = TMEM lane
     const int head_half = tid >> 6;                    // 0: head A, 1: head B
@@ -83,7 +86,7 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
     int hp_loaded = -1;
 
     constexpr uint32_t IDESC_S = umma_idesc_bf16(128, 128, false, false);
-    constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 64, false, true);
+    constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 32, false, true);
 
     auto coord_of = [&](int b, int i, int hp) -> TileCoord {
         TileCoord t;
@@ -94,63 +97,47 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
         t.c0 = hp * 64;
         return t;
     };
-    // byte offset of this thread's chunk of region r (image b, head pair's 64 channels at c0)
-    auto region_off = [&](int b, int r, int c0) -> size_t {
-        const int ry = (r * inv_s) >> 20, rx = r - ry * dm.S;
-        return (size_t)b * img_bytes + (size_t)(ry * RS) * row_bytes + (size_t)(rx * RS) * dm.C * 2 + (size_t)c0 * 2 + thr_off;
-    };
-    // routing entries (head A, head B) of a unit = (tile, routed step); -1: out of range.  The index may
-    // come from a kernel this one overlaps (programmatic dependent launch): coherent loads after
-    // pdl_wait(), never the read-only path, whose loads the compiler may move above the wait
-    auto read_entries = [&](const TileCoord& t, int m) -> int2 {
+    // routing entries (head A, head B) of a tile; -1: out of range.  The index may come from a kernel this
+    // one overlaps (programmatic dependent launch): coherent loads after pdl_wait(), never the read-only
+    // path, whose loads the compiler may move above the wait
+    auto read_entries = [&](const TileCoord& t) -> int2 {
         const int hA = 2 * t.hp, hB = hA + 1;
         const int hiA = dm.heads_i == 1 ? 0 : hA, hiB = dm.heads_i == 1 ? 0 : hB;
-        int ra = __ldcg(index + (((size_t)t.b * dm.heads_i + hiA) * dm.R + t.i) * dm.topk + m);
-        int rb = __ldcg(index + (((size_t)t.b * dm.heads_i + hiB) * dm.R + t.i) * dm.topk + m);
+        int ra = __ldcg(index + ((size_t)t.b * dm.heads_i + hiA) * dm.R + t.i);
+        int rb = __ldcg(index + ((size_t)t.b * dm.heads_i + hiB) * dm.R + t.i);
         if (ra < 0 || ra >= dm.R) { record_error(status, BRA_ERR_INDEX, ra); ra = -1; }
         if (rb < 0 || rb >= dm.R) { record_error(status, BRA_ERR_INDEX, rb); rb = -1; }
         return make_int2(ra, rb);
     };
-    auto load_k = [&](const TileCoord& t, int2 ent, int buf) {
-        int r = lhead ? ent.y : ent.x;
-        r = r < 0 ? 0 : r;                  // an invalid entry loads region 0; its P is zero
-        const uint8_t* src = Kb + region_off(t.b, r, t.c0);
-        const uint32_t kd = sm_base + (buf ? OFF_KV1 : OFF_K) + tile_off;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) cp_async_16(kd + i * 512, src + i * row_bytes, 16);
+    // ---- copies: issued by thread 0 only.  A box is named by (channel, x, y, image) of its first element.
+    // j: ordinal of the tile among this CTA's (its parity is the phase of the barrier); remembered so that
+    // a CTA that gives up can still wait for what it has in flight.
+    int last_qk = -1, last_v = -1, last_h = -1;
+    auto issue_qk = [&](const TileCoord& t, int2 ent, int j) {
+        last_qk = j;
+        const int ra = ent.x < 0 ? 0 : ent.x, rb = ent.y < 0 ? 0 : ent.y;   // an invalid entry loads region 0; its P is zero
+        const int rya = (ra * inv_s) >> 20, ryb = (rb * inv_s) >> 20;
+        mbar_expect_tx(bar_qk, k1::QK_BYTES);
+        tma_load_4d(sm_base + OFF_Q, &maps.q, bar_qk, t.c0, t.x0, t.y0, t.b);
+        tma_load_4d(sm_base + OFF_Q + 4096, &maps.q, bar_qk, t.c0 + 32, t.x0, t.y0, t.b);
+        tma_load_4d(sm_base + OFF_K, &maps.k, bar_qk, t.c0, (ra - rya * dm.S) * RS, rya * RS, t.b);
+        tma_load_4d(sm_base + OFF_K + 4096, &maps.k, bar_qk, t.c0 + 32, (rb - ryb * dm.S) * RS, ryb * RS, t.b);
     };
-    auto load_v = [&](const TileCoord& t, int2 ent, int buf) {
-        int r = lhead ? ent.y : ent.x;
-        r = r < 0 ? 0 : r;
-        const uint8_t* src = Vb + region_off(t.b, r, t.c0);
-        const uint32_t vd = sm_base + (buf ? OFF_KV1 + 8192 : OFF_V) + v_off;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) cp_async_16(vd + i * 1024, src + i * row_bytes, 16);
+    auto issue_v = [&](const TileCoord& t, int2 ent, int j) {
+        last_v = j;
+        const int ra = ent.x < 0 ? 0 : ent.x, rb = ent.y < 0 ? 0 : ent.y;
+        const int rya = (ra * inv_s) >> 20, ryb = (rb * inv_s) >> 20;
+        mbar_expect_tx(bar_v, k1::V_BYTES);
+        tma_load_4d(sm_base + OFF_V, &maps.v, bar_v, t.c0, (ra - rya * dm.S) * RS, rya * RS, t.b);
+        tma_load_4d(sm_base + k1::OFF_VB, &maps.v, bar_v, t.c0 + 32, (rb - ryb * dm.S) * RS, ryb * RS, t.b);
     };
-    auto load_q = [&](const TileCoord& t) {
-        const uint8_t* src = Qb + region_off(t.b, t.i, t.c0);
-        const uint32_t dst = sm_base + OFF_Q + tile_off;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) cp_async_16(dst + i * 512, src + i * row_bytes, 16);
+    auto issue_halo = [&](const TileCoord& t, int j) {
+        if (!dm.lce) return;
+        last_h = j;
+        mbar_expect_tx(bar_h, HALO_BYTES);
+        tma_load_4d(sm_base + OFF_HALO, &maps.halo, bar_h, t.c0, t.x0 - 2, t.y0 - 2, t.b);
     };
-    // halo: thread (column hx = tid >> 3 of the 12, 16-byte chunk c) copies its chunk of every one of the
-    // 12 halo rows; threads 96..127 have no column.  Zeros outside the map (the conv's zero padding).
-    const int hx = tid >> 3;
-    auto load_halo = [&](const TileCoord& t) {
-        if (!dm.lce || hx >= HALO) return;
-        const bool col_in = (t.x0 + hx >= 2) && (t.x0 + hx - 2 < dm.W);
-        const uint8_t* src = Vb + (size_t)t.b * img_bytes + (size_t)t.x0 * dm.C * 2 + (size_t)t.c0 * 2 + c * 16 +
-                             (ptrdiff_t)(hx - 2) * dm.C * 2;
-        const uint32_t hd = sm_base + OFF_HALO + tid * 16;
-#pragma unroll
-        for (int hy = 0; hy < HALO; ++hy) {
-            const int y = t.y0 + hy - 2;
-            const bool inb = col_in && y >= 0 && y < dm.H;
-            cp_async_16(hd + hy * (HALO * 128), inb ? src + (ptrdiff_t)y * (ptrdiff_t)row_bytes : Vb, inb ? 16u : 0u);
-        }
-    };
-
-    auto issue_s = [&]() {                  // one thread: S = Q K^T for the tile whose Q and K are in shared memory
+    auto issue_s = [&]() {                  // S = Q K^T for the tile whose Q and K are in shared memory
         tc_fence_after_sync();
         const uint32_t qa = sm_base + OFF_Q, ka = sm_base + OFF_K;
 #pragma unroll
@@ -162,25 +149,18 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
 
     bool ok = true;
     TileCoord t = coord_of(walk.b, walk.i, walk.hp);
-    // copies of a tile go out in three groups: (Q, K), then V, then the halo.
-    // Q is an input of the call: its copy (and everything above) overlaps the tail of the kernel before
-    // (routing, in a forward call); only the routing index has to wait for it
-    if (my_tiles > 0) load_q(t);
-    pdl_wait();
+    pdl_wait();                             // the routing index comes from the kernel before (a forward call)
     int2 ent = make_int2(0, 0);             // routing entries (head A, head B) of the tile in hand
     if (my_tiles > 0) {
-        ent = read_entries(t, 0);
-        load_k(t, ent, 0);
+        ent = read_entries(t);
+        if (tid == 0) {
+            issue_qk(t, ent, 0);
+            issue_v(t, ent, 0);
+            issue_halo(t, 0);
+            ok = mbar_wait(bar_qk, 0, POLL_LIMIT);
+            if (ok) issue_s();
+        }
     }
-    cp_async_commit();
-    if (my_tiles > 0) load_v(t, ent, 0);
-    cp_async_commit();
-    if (my_tiles > 0) load_halo(t);
-    cp_async_commit();
-    cp_async_wait<2>();
-    fence_proxy_async_smem();
-    __syncthreads();
-    if (tid == 0 && my_tiles > 0) issue_s();
 
     for (int n = 0; n < my_tiles; ++n) {
         if (dm.lce && t.hp != hp_loaded) {
@@ -194,15 +174,14 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
         if (has_next) walk.next();
         const TileCoord tn = has_next ? coord_of(walk.b, walk.i, walk.hp) : t;
         int2 ent_n = ent;
-        if (has_next) ent_n = read_entries(tn, 0);
+        if (has_next) ent_n = read_entries(tn);
+        const uint32_t par = n & 1;
 
-        // ---- S of this tile is in TMEM (issued a tile ago) ----
-        if (warp == 0) ok = mbar_wait(bar_s, n & 1, POLL_LIMIT);     // one warp polls, the rest sleep at the barrier
-        if (!__syncthreads_and(ok)) { ok = false; break; }
+        // ---- S of this tile is in TMEM (issued a tile ago); the MMA has read Q and K, so the next
+        // tile's take their place ----
+        ok = mbar_wait(bar_s, par, POLL_LIMIT) && ok;
         tc_fence_after_sync();
-        // the MMA has read Q and K: the next tile's take their place
-        if (has_next) { load_q(tn); load_k(tn, ent_n, 0); }
-        cp_async_commit();
+        if (tid == 0 && has_next && ok) issue_qk(tn, ent_n, n + 1);
 
         // ---- softmax: thread = row.  Pass 1: row maximum ----
         const bool valid = (head_half ? ent.y : ent.x) >= 0;
@@ -240,21 +219,24 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
             tmem_st_32x32b_x8(p_addr + (cc >> 1), pk);
         }
         tmem_st_wait();
-        // V and the halo of this tile have landed (the next tile's Q and K may still be in flight)
-        cp_async_wait<1>();
-        fence_proxy_async_smem();
         tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after_sync();
-            const uint64_t vd = umma_smem_desc(sm_base + OFF_V, 16, 1024, 2);
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)         // 64 keys = 4 k-steps of 16 (2048 B of V each)
-                umma_ts(tmem + TM_O, tmem + ks * 8, vd + (uint64_t)(ks * 128), IDESC_O, ks);
-            umma_commit(bar_o);
-        }
-        if (warp == 0) ok = mbar_wait(bar_o, n & 1, POLL_LIMIT);
         if (!__syncthreads_and(ok)) { ok = false; break; }
+        // ---- O = P V: head A's V tile gives columns 64..95, head B's 96..127; a row keeps its own head's ----
+        if (tid == 0) {
+            ok = mbar_wait(bar_v, par, POLL_LIMIT);
+            if (ok) {
+                tc_fence_after_sync();
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const uint64_t vd = umma_smem_desc(sm_base + (hh ? k1::OFF_VB : OFF_V), 16, 512, 4);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)     // 64 keys = 4 k-steps of 16 (1024 B of a V tile each)
+                        umma_ts(tmem + TM_O + hh * 32, tmem + ks * 8, vd + (uint64_t)(ks * 64), IDESC_O, ks);
+                }
+                umma_commit(bar_o);
+            }
+        }
+        ok = mbar_wait(bar_o, par, POLL_LIMIT) && ok;
         tc_fence_after_sync();
         // ---- normalise, stage O^att as fp32 [64 tokens][64 ch] (16-byte units xor-swizzled) ----
         {
@@ -275,12 +257,13 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
                 lse[((size_t)t.b * dm.heads + 2 * t.hp + head_half) * dm.N + (size_t)(t.y0 + tq / RS) * dm.W + t.x0 + tq % RS] =
                     (valid ? mx + log2f(l_run) : -INFINITY) * 0.6931471805599453f;
         }
-        // Q and K of the next tile have landed; TMEM has been read: the tensor core starts on the next tile
-        cp_async_wait<0>();
-        fence_proxy_async_smem();
+        // TMEM has been read: the tensor core starts on the next tile as soon as its Q and K have landed
         tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0 && has_next) issue_s();
+        if (!__syncthreads_and(ok)) { ok = false; break; }
+        if (tid == 0 && has_next) {
+            ok = mbar_wait(bar_qk, par ^ 1, POLL_LIMIT);
+            if (ok) issue_s();
+        }
 
         // ---- LCE + store ----
         // Input row yy of the halo feeds output rows yy - ti through tap row ti.  Fully unrolled:
@@ -297,10 +280,13 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
 #pragma unroll
                 for (int xx = 0; xx < 2; ++xx)
                     acc[y][xx] = __fadd2_rn(lds_f32x2(stage + (y * RS + xx) * 256 + (xx ? sw1 : sw0)), bias2);
-            __syncthreads();                // the staging tile has been read: V of the next tile takes its place
-            if (has_next) load_v(tn, ent_n, 0);
-            cp_async_commit();
+            // the staging tile has been read (by ordinary loads: fence before the bulk copy that overwrites
+            // it): V of the next tile takes its place
+            fence_proxy_async_smem();
+            __syncthreads();
+            if (tid == 0 && has_next && ok) issue_v(tn, ent_n, n + 1);
             if (dm.lce) {
+                ok = mbar_wait(bar_h, par, POLL_LIMIT) && ok;      // the halo of this tile has landed
 #pragma unroll
                 for (int yy = 0; yy < HALO; ++yy) {
                     float2 v[6];
@@ -332,18 +318,24 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
                 out += out_row;
             }
         }
-        __syncthreads();                    // the halo is free
-        if (has_next) load_halo(tn);
-        cp_async_commit();
+        fence_proxy_async_smem();
+        __syncthreads();                    // the halo has been read: the next tile's takes its place
+        if (tid == 0 && has_next && ok) issue_halo(tn, n + 1);
         t = tn;
         ent = ent_n;
     }
 
     // ---- teardown: nothing in flight, TMEM returned ----
-    cp_async_wait<0>();
     tc_fence_before_sync();
+    const bool all_ok = __syncthreads_and(ok);
+    if (tid == 0 && !all_ok) {
+        record_error(status, BRA_ERR_TIMEOUT, blockIdx.x);
+        // bounded waits for the copies this CTA still has in flight (immediate for those that have landed)
+        if (last_qk >= 0) mbar_wait(bar_qk, last_qk & 1, POLL_LIMIT);
+        if (last_v >= 0) mbar_wait(bar_v, last_v & 1, POLL_LIMIT);
+        if (last_h >= 0) mbar_wait(bar_h, last_h & 1, POLL_LIMIT);
+    }
     __syncthreads();
-    if (tid == 0 && !ok) record_error(status, BRA_ERR_TIMEOUT, blockIdx.x);
     if (warp == 0) {
         __syncwarp();
         tc_fence_after_sync();
@@ -352,6 +344,38 @@ attend_tc_k1_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* _
 }
 
 // ------------------------------------------------------------------ host side
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's encoder, looked up through the runtime (the library does not link against the driver).
+EncodeTiledFn encoder() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// Tensor map over a [B,H,W,C] bf16 tensor of this GPU's memory; box = (bc channels, bx, by tokens, 1 image).
+bool make_map(CUtensorMap* m, const void* base, const Dims& d, int bc, int bx, int by, CUtensorMapSwizzle sw) {
+    EncodeTiledFn enc = encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)d.C, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.B};
+    const cuuint64_t strides[3] = {(cuuint64_t)d.C * 2, (cuuint64_t)d.W * d.C * 2, (cuuint64_t)d.H * d.W * d.C * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)bc, (cuuint32_t)bx, (cuuint32_t)by, 1};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+}  // namespace
+
 cudaError_t launch_attend_tc_k1(const Dims& d, const void* Q, const void* K, const void* V,
                                 const int32_t* index, const float* lce_w, const float* lce_b,
                                 void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel) {
@@ -363,13 +387,17 @@ cudaError_t launch_attend_tc_k1(const Dims& d, const void* Q, const void* K, con
         return cudaFuncSetAttribute(attend_tc_k1_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     });
     if (e != cudaSuccess) return e;
+    K1Maps maps;
+    if (!make_map(&maps.q, Q, d, 32, tc::RS, tc::RS, CU_TENSOR_MAP_SWIZZLE_64B) ||
+        !make_map(&maps.k, K, d, 32, tc::RS, tc::RS, CU_TENSOR_MAP_SWIZZLE_64B) ||
+        !make_map(&maps.v, V, d, 32, tc::RS, tc::RS, CU_TENSOR_MAP_SWIZZLE_64B) ||
+        !make_map(&maps.halo, V, d, 64, tc::HALO, tc::HALO, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return cudaErrorInvalidValue;
     const int tiles = d.B * d.R * (d.heads / 2);
     const int resident = tc_sm_count() * 4;
     const unsigned grid = (unsigned)(tiles < resident ? tiles : resident);
     e = launch_kernel(attend_tc_k1_kernel, dim3(grid), dim3(tc::THREADS), tc::SMEM_K1, st, after_own_kernel,
-                      static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
-                      static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b,
-                      static_cast<__nv_bfloat16*>(O), lse, status, d, tiles);
+                      maps, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, tiles);
     count_launch();
     return e;
 }

@@ -1,8 +1,10 @@
 // Thin inline-PTX wrappers for the sm_100a features the kernels use:
-// mbarrier, 16-byte asynchronous copies (cp.async), tcgen05 MMA / TMEM.
+// mbarrier, 16-byte asynchronous copies (cp.async), bulk tensor copies (TMA, this GPU's memory only,
+// never multicast), tcgen05 MMA / TMEM.
 // Every wait is bounded: it returns false once its poll budget is spent.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -46,6 +48,11 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void fence_mbar_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
+// One arrival that also announces `bytes` of bulk-copy data to come (the phase completes once they have landed).
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -81,6 +88,17 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// ---------------------------------------------------------------- TMA
+// 4-D tiled load global -> this CTA's shared memory; coordinates innermost first.  c0 * element size must
+// be a multiple of 16 bytes; the other coordinates may lie outside the tensor (the fill value is written).
+__device__ __forceinline__ void tma_load_4d(uint32_t dst_smem, const CUtensorMap* map, uint64_t* bar,
+                                            int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
 }
 
 // ---------------------------------------------------------------- proxies / fences
