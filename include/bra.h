@@ -73,8 +73,9 @@ typedef enum bra_impl {
     BRA_IMPL_IMG = 4,   /* bf16 warp-level tensor-core kernel with a whole (image, head) of K and V resident in
                            shared memory (C/heads == 32, H*W <= ~1500 tokens): small maps, small regions */
     BRA_IMPL_TC_FUSED = 5 /* as BRA_IMPL_TC, and bra_forward runs pooling, routing and attention in ONE launch
-                           (8 x 8-token regions, topk = 1, per-head routing, <= 64 regions, C <= 128); never
-                           chosen by BRA_IMPL_AUTO: on B200 the chain of three launches is faster */
+                           (8 x 8-token regions, topk = 1, per-head routing, <= 64 regions, C <= 128): same index
+                           bit for bit, O and lse equal up to summation order; never chosen by BRA_IMPL_AUTO:
+                           on B200 the chain of three launches is faster */
 } bra_impl;
 
 /*

@@ -100,14 +100,18 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
     // routing entries (head A, head B) of a tile; -1: out of range.  The index may come from a kernel this
     // one overlaps (programmatic dependent launch): coherent loads after pdl_wait(), never the read-only
     // path, whose loads the compiler may move above the wait
-    auto read_entries = [&](const TileCoord& t) -> int2 {
-        const int hA = 2 * t.hp, hB = hA + 1;
+    // The loads are issued two tiles ahead of the tile they serve and looked at (checked) one tile later,
+    // so that their latency is never waited for.
+    auto load_entries = [&](int b, int i, int hp) -> int2 {
+        const int hA = 2 * hp, hB = hA + 1;
         const int hiA = dm.heads_i == 1 ? 0 : hA, hiB = dm.heads_i == 1 ? 0 : hB;
-        int ra = __ldcg(index + ((size_t)t.b * dm.heads_i + hiA) * dm.R + t.i);
-        int rb = __ldcg(index + ((size_t)t.b * dm.heads_i + hiB) * dm.R + t.i);
-        if (ra < 0 || ra >= dm.R) { record_error(status, BRA_ERR_INDEX, ra); ra = -1; }
-        if (rb < 0 || rb >= dm.R) { record_error(status, BRA_ERR_INDEX, rb); rb = -1; }
-        return make_int2(ra, rb);
+        return make_int2(__ldcg(index + ((size_t)b * dm.heads_i + hiA) * dm.R + i),
+                         __ldcg(index + ((size_t)b * dm.heads_i + hiB) * dm.R + i));
+    };
+    auto checked = [&](int2 e) -> int2 {
+        if (e.x < 0 || e.x >= dm.R) { record_error(status, BRA_ERR_INDEX, e.x); e.x = -1; }
+        if (e.y < 0 || e.y >= dm.R) { record_error(status, BRA_ERR_INDEX, e.y); e.y = -1; }
+        return e;
     };
     // ---- copies: issued by thread 0 only.  A box is named by (channel, x, y, image) of its first element.
     // j: ordinal of the tile among this CTA's (its parity is the phase of the barrier); remembered so that
@@ -151,8 +155,14 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
     TileCoord t = coord_of(walk.b, walk.i, walk.hp);
     pdl_wait();                             // the routing index comes from the kernel before (a forward call)
     int2 ent = make_int2(0, 0);             // routing entries (head A, head B) of the tile in hand
+    int2 raw_n = make_int2(0, 0);           // those of the next tile, as loaded (not yet looked at)
+    if (my_tiles > 1) {
+        walk.next();                        // the walker stays one tile ahead of `tn`
+        raw_n = load_entries(walk.b, walk.i, walk.hp);
+    }
+    TileCoord tn = my_tiles > 1 ? coord_of(walk.b, walk.i, walk.hp) : t;
     if (my_tiles > 0) {
-        ent = read_entries(t);
+        ent = checked(load_entries(t.b, t.i, t.hp));
         if (tid == 0) {
             issue_qk(t, ent, 0);
             issue_v(t, ent, 0);
@@ -171,10 +181,11 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
             hp_loaded = t.hp;
         }
         const bool has_next = n + 1 < my_tiles;
-        if (has_next) walk.next();
-        const TileCoord tn = has_next ? coord_of(walk.b, walk.i, walk.hp) : t;
-        int2 ent_n = ent;
-        if (has_next) ent_n = read_entries(tn);
+        const int2 ent_n = has_next ? checked(raw_n) : ent;       // loaded a tile ago
+        if (n + 2 < my_tiles) {
+            walk.next();
+            raw_n = load_entries(walk.b, walk.i, walk.hp);         // for the tile after next
+        }
         const uint32_t par = n & 1;
 
         // ---- S of this tile is in TMEM (issued a tile ago); the MMA has read Q and K, so the next
@@ -183,40 +194,48 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
         tc_fence_after_sync();
         if (tid == 0 && has_next && ok) issue_qk(tn, ent_n, n + 1);
 
-        // ---- softmax: thread = row.  Pass 1: row maximum ----
+        // ---- softmax: thread = row.  Loads from tensor memory are issued one step ahead of their use.
+        // Pass 1: row maximum, 32 columns at a time ----
         const bool valid = (head_half ? ent.y : ent.x) >= 0;
-        float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll 1
-        for (int cc = 0; cc < 64; cc += 16) {
-            uint32_t r[16];
-            tmem_ld_32x32b_x16(s_addr + cc, r);
-            tmem_ld_wait();
+        float mx;
+        {
+            float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-            for (int q = 0; q < 16; q += 4) {
-                m0 = fmax3(m0, __uint_as_float(r[q]), __uint_as_float(r[q + 1]));
-                m1 = fmax3(m1, __uint_as_float(r[q + 2]), __uint_as_float(r[q + 3]));
+            for (int half = 0; half < 2; ++half) {
+                uint32_t ra[32];
+                tmem_ld_32x32b_x32(s_addr + 32 * half, ra);
+                tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 32; q += 4) {
+                    m0 = fmax3(m0, __uint_as_float(ra[q]), __uint_as_float(ra[q + 1]));
+                    m1 = fmax3(m1, __uint_as_float(ra[q + 2]), __uint_as_float(ra[q + 3]));
+                }
             }
+            mx = fmaxf(m0, m1) * sl2;                                  // sl2 > 0
         }
-        const float mx = fmaxf(m0, m1) * sl2;                          // sl2 > 0
         // an out-of-range routing entry: every probability of the row is exp2(-inf) = 0
         const float mneg = valid ? -mx : -INFINITY;
         // pass 2: P = exp2(S * scale * log2 e - max), bf16 pairs written over the columns
         // of S already consumed (column j of P never outruns column 2j of S); row sum
         const float2 sl2v = make_float2(valid ? sl2 : 0.f, valid ? sl2 : 0.f), mnegv = make_float2(mneg, mneg);
         float2 sum2 = make_float2(0.f, 0.f);
-#pragma unroll 1
-        for (int cc = 0; cc < 64; cc += 16) {
-            uint32_t r[16], pk[8];
-            tmem_ld_32x32b_x16(s_addr + cc, r);
-            tmem_ld_wait();
+        {
+            uint32_t r[2][16];
+            tmem_ld_32x32b_x16(s_addr, r[0]);
 #pragma unroll
-            for (int q = 0; q < 16; q += 2) {
-                const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[q]), __uint_as_float(r[q + 1])), sl2v, mnegv);
-                const float2 pe = make_float2(ex2f(a.x), ex2f(a.y));
-                sum2 = __fadd2_rn(sum2, pe);
-                pk[q >> 1] = pack_bf16(pe.x, pe.y);
+            for (int ch = 0; ch < 4; ++ch) {
+                tmem_ld_wait();
+                if (ch < 3) tmem_ld_32x32b_x16(s_addr + 16 * (ch + 1), r[(ch + 1) & 1]);
+                uint32_t pk[8];
+#pragma unroll
+                for (int q = 0; q < 16; q += 2) {
+                    const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[ch & 1][q]), __uint_as_float(r[ch & 1][q + 1])), sl2v, mnegv);
+                    const float2 pe = make_float2(ex2f(a.x), ex2f(a.y));
+                    sum2 = __fadd2_rn(sum2, pe);
+                    pk[q >> 1] = pack_bf16(pe.x, pe.y);
+                }
+                tmem_st_32x32b_x8(p_addr + 8 * ch, pk);
             }
-            tmem_st_32x32b_x8(p_addr + (cc >> 1), pk);
         }
         tmem_st_wait();
         tc_fence_before_sync();
@@ -323,6 +342,7 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
         if (tid == 0 && has_next && ok) issue_halo(tn, n + 1);
         t = tn;
         ent = ent_n;
+        if (n + 2 < my_tiles) tn = coord_of(walk.b, walk.i, walk.hp);
     }
 
     // ---- teardown: nothing in flight, TMEM returned ----
