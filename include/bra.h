@@ -25,8 +25,8 @@
  *     p->shared_routing != 0).  Row i lists the key regions that the queries of
  *     region i attend to.  It is a list: any order, duplicates count twice.
  *   - ws: scratch of at least bra_workspace_bytes(p) bytes, 256-byte aligned.
- *     It holds a device status block and, for the one-launch forward, job
- *     counters and per-image flags that the kernels expect to find ZERO and
+ *     It holds a device status block (error words and, for the one-launch
+ *     forward, barrier counters) that the kernels expect to find ZERO and
  *     leave zero: before its first use fill ws with zeros or call
  *     bra_workspace_init().  bra_device_status() restores that state when it
  *     reports an error.  Calls that share a ws must be ordered on one stream.
@@ -72,18 +72,18 @@ typedef enum bra_impl {
     BRA_IMPL_TC = 3,    /* bf16 tcgen05/TMEM kernels (C/heads == 32; regions of 8 x 8 tokens, or 16 wide and a multiple of 8 high) */
     BRA_IMPL_IMG = 4,   /* bf16 warp-level tensor-core kernel with a whole (image, head) of K and V resident in
                            shared memory (C/heads == 32, H*W <= ~1500 tokens): small maps, small regions */
-    BRA_IMPL_TC_FUSED = 5 /* as BRA_IMPL_TC, and bra_forward runs pooling, routing and attention in ONE launch
-                           (8 x 8-token regions, topk = 1, per-head routing, <= 64 regions, C <= 128): same index
-                           bit for bit, O and lse equal up to summation order; never chosen by BRA_IMPL_AUTO:
-                           on B200 the chain of three launches is faster */
+    BRA_IMPL_TC_FUSED = 5 /* as BRA_IMPL_TC, and bra_forward runs pooling, routing and attention as three phases of
+                           ONE launch (8 x 8-token regions, topk = 1, per-head routing, <= 64 regions,
+                           C <= 128): results equal to the chain of launches bit for bit */
 } bra_impl;
 
 /*
  * Failure injection for tests of the error path (no GPU fault, trap or hang is involved).
- * BRA_INJECT_HOLD_ROUTE_FLAGS: in the one-launch forward (bra_forward with BRA_IMPL_TC_FUSED) the
- * routing step keeps the per-image "routed" flags down, so every attention job's bounded
- * wait on them runs out after a few thousand polls with no tensor-core work in flight; the kernel returns
- * normally, O is not written and bra_device_status() reports BRA_ERR_TIMEOUT.  Ignored by every other path.
+ * BRA_INJECT_HOLD_ROUTE_FLAGS: in the one-launch forward (bra_forward with BRA_IMPL_TC_FUSED) one pooled
+ * unit is never counted as done, so every CTA's bounded wait for the end of the pooling phase runs out
+ * after a few thousand polls, before any tensor-core work or tile copy has been issued;
+ * the kernel returns normally, O is not written and bra_device_status() reports BRA_ERR_TIMEOUT.
+ * Ignored by every other path.
  */
 typedef enum bra_inject { BRA_INJECT_NONE = 0, BRA_INJECT_HOLD_ROUTE_FLAGS = 1 } bra_inject;
 
@@ -106,8 +106,8 @@ typedef struct bra_problem {
 size_t bra_workspace_bytes(const bra_problem* p);
 
 /*
- * Puts ws into the state the kernels expect: status block, job counters and per-image flags zero
- * (asynchronous memsets on `stream`; the rest of ws needs no initial value).  Needed once before the
+ * Puts ws into the state the kernels expect: status block (error words, barrier counters) zero
+ * (an asynchronous memset on `stream`; the rest of ws needs no initial value).  Needed once before the
  * first use of a ws that was not zero-filled.  (Housekeeping of this library: Algorithm 1 has no
  * counterpart.)
  */
@@ -209,7 +209,7 @@ bra_status bra_backward(const bra_problem* p, const void* Q, const void* K, cons
  * Synchronises `stream`, then returns and clears the first device-detected
  * error recorded in ws (BRA_OK, BRA_ERR_INDEX, BRA_ERR_TIMEOUT, or BRA_ERR_CUDA
  * if the synchronisation itself failed).  When it reports an error it also puts the
- * counters and flags in ws back to zero (as bra_workspace_init does), so the next call
+ * barrier counters in ws back to zero (as bra_workspace_init does), so the next call
  * starts clean.  ws must have been initialised and used by an earlier call.
  */
 bra_status bra_device_status(void* ws, void* stream);

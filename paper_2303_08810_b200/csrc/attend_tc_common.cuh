@@ -23,7 +23,7 @@ constexpr int OFF_Q = 0;                                 // [128 rows][64 B]  64
 constexpr int OFF_K = 8192;                              // [128 keys][64 B]  64B swizzle, K-major (buffer 0)
 constexpr int OFF_V = 16384;                             // [64 keys][128 B]  128B swizzle, MN-major (buffer 0)
 constexpr int OFF_ST = OFF_V;                            // [64 tokens][64 ch] fp32 staging: over V (buffer 0) + scratch
-constexpr int OFF_POOL = 24576;                          // 8 KB scratch of the fused forward: pooling partial sums, K^r of a head
+constexpr int OFF_POOL = 24576;                          // second half of the staging tile; scratch of the one-launch forward (pooling partial sums, K^r of a head)
 constexpr int OFF_HALO = 32768;                          // [12][12][64 ch] bf16, linear
 constexpr int OFF_BAR = OFF_HALO + HALO_BYTES;           // 51200: two mbarriers, tmem slot, job slots
 constexpr int OFF_MISC = OFF_BAR + 64;                   // 1 KB: routing step, best key per (half, row)
@@ -32,8 +32,7 @@ constexpr int SMEM_K1 = OFF_MISC + 1024 + 1024;          // + slack for the manu
 constexpr int SMEM_KN = OFF_KV1 + 16384 + 1024;
 static_assert(OFF_KV1 % 1024 == 0 && OFF_KV1 >= OFF_MISC + 1024, "buffer 1 placement");
 constexpr uint32_t POLL_LIMIT = 4000000u;
-constexpr uint32_t FLAG_POLLS = 1u << 20;                // x ~0.1-0.5 us per poll: a fraction of a second
-constexpr int FUSED_MAX_R = 64;                          // routing step: one thread per (row, half of the candidates)
+constexpr uint32_t FLAG_POLLS = 1u << 20;                // polls of a grid-wide barrier, x ~0.2-0.5 us each: a fraction of a second
 }  // namespace tc
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -66,11 +65,6 @@ __device__ __forceinline__ uint32_t score_bits(float s) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-#ifndef BRA_TR
-#define BRA_TR(n, ev) do { } while (0)
-#define BRA_CNT(i, v) do { } while (0)
-#endif
-
 struct TileCoord { int b, i, hp, y0, x0, c0; };
 // Walks tiles T, T + stride, ... (T = (b * R + i) * pairs + hp) with adds and carries only.
 struct TileWalker {
@@ -92,22 +86,6 @@ struct TileWalker {
         b += d_b + carry;
     }
 };
-
-// What the fused forward adds to the arguments of the attention kernel.
-struct FusedArgs {
-    float* q_mean;          // [B,R,C] Q^r (scratch)
-    float* k_mean;          // [B,R,C] K^r (scratch)
-    int32_t* index_out;     // [B,heads,R,1] written by the routing step, read by the attention part
-    int32_t* pool_cnt;      // [B] units of image b pooled so far        } zero at launch,
-    int32_t* route_flag;    // [B] 1 once the index of image b is written  } zeroed again by the last CTA
-    int32_t* ctrl;          // status block: [8] job counter, [9] finished CTAs (same rule)
-    int delta;              // images the pooling runs ahead of the attention
-    int units;              // R * head pairs: jobs per image slot
-    int total;              // (B + delta) * units jobs
-    int inject;             // failure injection of the tests: 1 = the flags are never raised
-    int sync_off, sync_bytes;   // where pool_cnt / route_flag sit in the scratch buffer (recorded in ctrl[2], ctrl[3])
-};
-struct Job { int att_b, pool_b, i, hp; };      // image of the attention / pooling part (-1: none), region, head pair
 
 // the topk = 1 kernel (attend_tc_k1.cu); launch_attend_tc() forwards to it
 cudaError_t launch_attend_tc_k1(const Dims& d, const void* Q, const void* K, const void* V,

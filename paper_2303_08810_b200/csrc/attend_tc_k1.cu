@@ -31,13 +31,186 @@ constexpr int OFF_VB = tc::OFF_V + 4096;        // head B's V tile ([64 keys][64
 constexpr uint32_t QK_BYTES = 16384, V_BYTES = 8192;
 }  // namespace k1
 
+// ------------------------------------------------------------------ the forward pass in one launch
+// What the one-launch forward adds to the arguments of the attention kernel.  The grid runs three phases:
+// region pooling of Q and K, routing (Eq. 4, Eq. 5 with k = 1), then the attention above.  The work of the
+// first two phases is handed out by ticket counters and a phase is over when a completion counter has
+// reached the number of its work items: CTAs that are running do all of it, so progress never depends on
+// how many CTAs of the grid are resident (and every wait is bounded all the same).  Pooling and routing add
+// their terms in the order of the stand-alone kernels, so the index equals bra_route's bit for bit.
+struct FwdArgs {
+    const uint8_t* Q;       // [B,H,W,C] bf16
+    const uint8_t* K;
+    float* q_mean;          // [B,R,C] Q^r (scratch)
+    float* k_mean;          // [B,R,C] K^r (scratch)
+    int32_t* index_out;     // [B,heads,R,1]
+    int32_t* ctrl;          // status block; [8] pooling tickets, [9] pooled units, [10] routing tickets, [11] routed
+                            // items, [12] finished CTAs: zero at launch, put back to zero by the last CTA
+    int inject;             // failure injection of the tests: 1 = the first pooled unit is never counted
+};
+
+// Bounded wait until *ctr has reached target (all threads return the same answer).
+__device__ __noinline__ bool wait_count(const int32_t* ctr, int target, uint32_t polls) {
+    bool ok = true;
+    if (threadIdx.x == 0) {
+        ok = false;
+        for (uint32_t it = 0; it < polls; ++it) {
+            if (ld_acquire_gpu(ctr) >= target) { ok = true; break; }
+            __nanosleep(it < 32 ? 20 : 200);
+        }
+    }
+    return __syncthreads_and(ok);
+}
+
+// Phase 1: per-region average of Q and K (Section 3.2).  A unit is (image, region, 64-channel slab); thread
+// (row half, column, 16-byte channel vector) sums its four token rows in order, then one thread per channel
+// adds, column by column, (lower half + upper half): the order of the stand-alone kernel for 8-row regions.
+// The loads of the next unit fly while this one is reduced; its ticket was drawn a unit earlier.
+__device__ __noinline__ void forward_pool_phase(const FwdArgs& fw, const Dims& dm, uint8_t* smem) {
+    using namespace tc;
+    const int tid = threadIdx.x;
+    const int c = tid & 7, tx = (tid >> 3) & 7, yh = tid >> 6;
+    const int pairs = dm.heads >> 1;
+    const int units = dm.B * dm.R * pairs;
+    const size_t row_bytes = (size_t)dm.W * dm.C * 2;
+    const uint32_t part = smem_u32(smem) + OFF_POOL;         // [tensor][row half][column][64 ch] fp32
+    volatile int* slot = reinterpret_cast<volatile int*>(smem + OFF_MISC);
+    auto unit_off = [&](int u) -> size_t {
+        const int hp = u % pairs, r = (u / pairs) % dm.R, b = u / (pairs * dm.R);
+        const int ry = r / dm.S, rx = r - ry * dm.S;
+        return (size_t)b * dm.H * row_bytes + (size_t)(ry * RS + 4 * yh) * row_bytes + (size_t)(rx * RS + tx) * dm.C * 2 +
+               (size_t)hp * 128 + c * 16;
+    };
+    auto load_unit = [&](int u, uint4 (&v)[8]) {
+        const size_t off = unit_off(u);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { v[q] = ldg_nc_u4(fw.Q + off + q * row_bytes); v[4 + q] = ldg_nc_u4(fw.K + off + q * row_bytes); }
+    };
+    if (tid == 0) { slot[0] = atomicAdd(fw.ctrl + 8, 1); slot[1] = atomicAdd(fw.ctrl + 8, 1); }
+    __syncthreads();
+    int cur = slot[0], nxt = slot[1];
+    __syncthreads();
+    uint4 pv[8];
+    int done = 0;                                           // units this CTA has pooled: counted in one go at the end
+    if (cur < units) load_unit(cur, pv);
+    while (cur < units) {
+        int t2 = 0;
+        if (tid == 0) t2 = atomicAdd(fw.ctrl + 8, 1);       // the unit after next
+        uint4 nx[8];
+        if (nxt < units) load_unit(nxt, nx);
+#pragma unroll
+        for (int tsr = 0; tsr < 2; ++tsr) {
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint4 v = pv[4 * tsr + q];
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    acc[2 * e] += __uint_as_float(w[e] << 16);
+                    acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+                }
+            }
+            const uint32_t dst = part + ((((tsr * 2 + yh) * 8 + tx) * 64 + c * 8) << 2);
+            sts_f32x4(dst, acc[0], acc[1], acc[2], acc[3]);
+            sts_f32x4(dst + 16, acc[4], acc[5], acc[6], acc[7]);
+        }
+        __syncthreads();
+        {
+            const int tsr = tid >> 6, ch = tid & 63;
+            const uint32_t src = part + (((tsr * 2) * 8 * 64 + ch) << 2);
+            float s = 0.f;
+#pragma unroll
+            for (int x = 0; x < 8; ++x) s += lds_f32(src + x * 256) + lds_f32(src + 8 * 256 + x * 256);
+            const int hp = cur % pairs, r = (cur / pairs) % dm.R, b = cur / (pairs * dm.R);
+            float* dst = tsr ? fw.k_mean : fw.q_mean;
+            dst[((size_t)b * dm.R + r) * dm.C + hp * 64 + ch] = s * (1.0f / 64.0f);
+        }
+        if (tid == 0) slot[0] = t2;
+        __syncthreads();
+        if (!(fw.inject && cur == 0)) ++done;
+        cur = nxt;
+        nxt = slot[0];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) pv[q] = nx[q];
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0 && done) atomicAdd(fw.ctrl + 9, done);
+}
+
+// Phase 2: Eq. 4 and Eq. 5 (k = 1).  An item is (image, head, chunk of 16 affinity rows); K^r of the head
+// sits in shared memory as [R][8 x 16 B] with unit (c4 + j) & 7 of row j holding channels 4 c4..4 c4+3
+// (conflict-free for 16-byte reads by eight consecutive rows).  Thread = (row, one of eight candidate
+// classes j mod 8); each dot product adds its 32 channels in increasing order, as the stand-alone routing
+// kernels do; the best (score, lower region first) of the eight classes is found with shuffles.
+__device__ __noinline__ void forward_route_phase(const FwdArgs& fw, const Dims& dm, uint8_t* smem) {
+    using namespace tc;
+    const int tid = threadIdx.x;
+    const uint32_t ks = smem_u32(smem) + OFF_POOL;
+    volatile int* slot = reinterpret_cast<volatile int*>(smem + OFF_MISC);
+    const int chunks = (dm.R + 15) >> 4;
+    const int items = dm.B * dm.heads * chunks;
+    const int l8 = tid & 7, lrow = tid >> 3;
+    for (;;) {
+        if (tid == 0) slot[0] = atomicAdd(fw.ctrl + 10, 1);
+        __syncthreads();
+        const int it = slot[0];
+        if (it >= items) break;
+        const int ch = it % chunks, h = (it / chunks) % dm.heads, b = it / (chunks * dm.heads);
+        const float* kb = fw.k_mean + (size_t)b * dm.R * dm.C + h * 32;
+        for (int e = tid; e < dm.R * 8; e += THREADS) {
+            const int j = e >> 3, c4 = e & 7;
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(kb + (size_t)j * dm.C) + c4);
+            sts_f32x4(ks + ((j * 8 + ((c4 + j) & 7)) << 4), v.x, v.y, v.z, v.w);
+        }
+        const int i = ch * 16 + lrow;
+        const bool live = i < dm.R;
+        float4 q[8];
+        {
+            const float4* qrow = reinterpret_cast<const float4*>(fw.q_mean + ((size_t)b * dm.R + (live ? i : 0)) * dm.C + h * 32);
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4) q[c4] = __ldcg(qrow + c4);
+        }
+        __syncthreads();
+        unsigned long long best = 0ull;
+        for (int j = l8; j < dm.R; j += 8) {
+            float acc = 0.f;
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4) {
+                const float4 k4 = lds_f32x4(ks + ((j * 8 + ((c4 + j) & 7)) << 4));
+                acc = fmaf(q[c4].x, k4.x, acc);
+                acc = fmaf(q[c4].y, k4.y, acc);
+                acc = fmaf(q[c4].z, k4.z, acc);
+                acc = fmaf(q[c4].w, k4.w, acc);
+            }
+            const unsigned long long key = ((unsigned long long)score_bits(acc) << 32) | (0xffffffffu - (uint32_t)j);
+            best = key > best ? key : best;
+        }
+#pragma unroll
+        for (int sh = 1; sh < 8; sh <<= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, sh);
+            best = other > best ? other : best;
+        }
+        if (l8 == 0 && live)
+            fw.index_out[((size_t)b * dm.heads + h) * dm.R + i] = (int32_t)(0xffffffffu - (uint32_t)best);
+        __threadfence();
+        __syncthreads();                    // index written; K^r of the next item may take the place of this one
+        if (tid == 0) atomicAdd(fw.ctrl + 11, 1);
+    }
+}
+
 struct K1Maps { CUtensorMap q, k, v, halo; };   // {32 ch, 8, 8} boxes of Q, K, V; {64 ch, 12, 12} box of V
 
+// FORWARD: pooling and routing run first, in this launch (see FwdArgs).
+template <bool FORWARD>
 __global__ void __launch_bounds__(tc::THREADS, 4)
 attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
                     const float* __restrict__ lce_w, const float* __restrict__ lce_b,
                     __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
-                    int32_t* __restrict__ status, Dims dm, int num_tiles) {
+                    int32_t* __restrict__ status, Dims dm, int num_tiles, FwdArgs fw) {
     using namespace tc;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -153,15 +326,26 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
 
     bool ok = true;
     TileCoord t = coord_of(walk.b, walk.i, walk.hp);
-    pdl_wait();                             // the routing index comes from the kernel before (a forward call)
+    if (FORWARD) {
+        const uint32_t polls = fw.inject ? 2048u : FLAG_POLLS;
+        forward_pool_phase(fw, dm, smem);
+        ok = wait_count(fw.ctrl + 9, dm.B * dm.R * (dm.heads >> 1), polls);
+        if (ok) {
+            forward_route_phase(fw, dm, smem);
+            ok = wait_count(fw.ctrl + 11, dm.B * dm.heads * ((dm.R + 15) >> 4), polls);
+        }
+    } else {
+        pdl_wait();                         // the routing index comes from the kernel before (a forward call)
+    }
     int2 ent = make_int2(0, 0);             // routing entries (head A, head B) of the tile in hand
     int2 raw_n = make_int2(0, 0);           // those of the next tile, as loaded (not yet looked at)
+    const int run_tiles = ok ? my_tiles : 0;    // a barrier that gave up: no tile is started
     if (my_tiles > 1) {
         walk.next();                        // the walker stays one tile ahead of `tn`
         raw_n = load_entries(walk.b, walk.i, walk.hp);
     }
     TileCoord tn = my_tiles > 1 ? coord_of(walk.b, walk.i, walk.hp) : t;
-    if (my_tiles > 0) {
+    if (run_tiles > 0) {
         ent = checked(load_entries(t.b, t.i, t.hp));
         if (tid == 0) {
             issue_qk(t, ent, 0);
@@ -172,7 +356,7 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
         }
     }
 
-    for (int n = 0; n < my_tiles; ++n) {
+    for (int n = 0; n < run_tiles; ++n) {
         if (dm.lce && t.hp != hp_loaded) {
             const float* wp = lce_w + (size_t)(t.c0 + 2 * lane) * 25;
 #pragma unroll
@@ -361,6 +545,14 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
+    if (FORWARD && tid == 0) {
+        // the last CTA to finish puts the counters back to zero for the next call
+        __threadfence();
+        if (atomicAdd(fw.ctrl + 12, 1) == (int)gridDim.x - 1 && all_ok) {
+#pragma unroll
+            for (int q = 8; q <= 12; ++q) fw.ctrl[q] = 0;
+        }
+    }
 }
 
 // ------------------------------------------------------------------ host side
@@ -396,28 +588,63 @@ bool make_map(CUtensorMap* m, const void* base, const Dims& d, int bc, int bx, i
 }
 }  // namespace
 
+static cudaError_t k1_attributes() {
+    static PerDeviceOnce once;
+    return once.run([]() -> cudaError_t {
+        cudaError_t a;
+        if ((a = cudaFuncSetAttribute(attend_tc_k1_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_K1)) != cudaSuccess) return a;
+        if ((a = cudaFuncSetAttribute(attend_tc_k1_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_K1)) != cudaSuccess) return a;
+        // several CTAs per SM: ask for the largest shared-memory carve-out
+        if ((a = cudaFuncSetAttribute(attend_tc_k1_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return a;
+        return cudaFuncSetAttribute(attend_tc_k1_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    });
+}
+
+static bool k1_maps(K1Maps* maps, const Dims& d, const void* Q, const void* K, const void* V) {
+    return make_map(&maps->q, Q, d, 32, tc::RS, tc::RS, CU_TENSOR_MAP_SWIZZLE_64B) &&
+           make_map(&maps->k, K, d, 32, tc::RS, tc::RS, CU_TENSOR_MAP_SWIZZLE_64B) &&
+           make_map(&maps->v, V, d, 32, tc::RS, tc::RS, CU_TENSOR_MAP_SWIZZLE_64B) &&
+           make_map(&maps->halo, V, d, 64, tc::HALO, tc::HALO, CU_TENSOR_MAP_SWIZZLE_NONE);
+}
+
 cudaError_t launch_attend_tc_k1(const Dims& d, const void* Q, const void* K, const void* V,
                                 const int32_t* index, const float* lce_w, const float* lce_b,
                                 void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel) {
-    static PerDeviceOnce once;
-    cudaError_t e = once.run([]() -> cudaError_t {
-        cudaError_t a = cudaFuncSetAttribute(attend_tc_k1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_K1);
-        if (a != cudaSuccess) return a;
-        // several CTAs per SM: ask for the largest shared-memory carve-out
-        return cudaFuncSetAttribute(attend_tc_k1_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    });
+    cudaError_t e = k1_attributes();
     if (e != cudaSuccess) return e;
     K1Maps maps;
-    if (!make_map(&maps.q, Q, d, 32, tc::RS, tc::RS, CU_TENSOR_MAP_SWIZZLE_64B) ||
-        !make_map(&maps.k, K, d, 32, tc::RS, tc::RS, CU_TENSOR_MAP_SWIZZLE_64B) ||
-        !make_map(&maps.v, V, d, 32, tc::RS, tc::RS, CU_TENSOR_MAP_SWIZZLE_64B) ||
-        !make_map(&maps.halo, V, d, 64, tc::HALO, tc::HALO, CU_TENSOR_MAP_SWIZZLE_NONE))
-        return cudaErrorInvalidValue;
+    if (!k1_maps(&maps, d, Q, K, V)) return cudaErrorInvalidValue;
     const int tiles = d.B * d.R * (d.heads / 2);
     const int resident = tc_sm_count() * 4;
     const unsigned grid = (unsigned)(tiles < resident ? tiles : resident);
-    e = launch_kernel(attend_tc_k1_kernel, dim3(grid), dim3(tc::THREADS), tc::SMEM_K1, st, after_own_kernel,
-                      maps, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, tiles);
+    e = launch_kernel(attend_tc_k1_kernel<false>, dim3(grid), dim3(tc::THREADS), tc::SMEM_K1, st, after_own_kernel,
+                      maps, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, tiles, FwdArgs{});
+    count_launch();
+    return e;
+}
+
+// The forward pass in one launch: per-head routing with k = 1, at most 64 regions, and a channel
+// count for which the stand-alone pooling kernel sums in the same order (so that the index equals bra_route's).
+bool forward_tc_supported(const Dims& d, int dtype) {
+    return attend_tc_supported(d, dtype) && d.topk == 1 && d.heads_i == d.heads && d.R <= 64 && d.C <= 128;
+}
+
+cudaError_t launch_forward_tc(const Dims& d, const void* Q, const void* K, const void* V,
+                              const float* lce_w, const float* lce_b, void* O, int32_t* index, float* lse,
+                              float* q_mean, float* k_mean, int32_t* ctrl, int inject, cudaStream_t st) {
+    cudaError_t e = k1_attributes();
+    if (e != cudaSuccess) return e;
+    K1Maps maps;
+    if (!k1_maps(&maps, d, Q, K, V)) return cudaErrorInvalidValue;
+    const int tiles = d.B * d.R * (d.heads / 2);
+    const int resident = tc_sm_count() * 4;
+    const unsigned grid = (unsigned)(tiles < resident ? tiles : resident);
+    FwdArgs fw;
+    fw.Q = static_cast<const uint8_t*>(Q); fw.K = static_cast<const uint8_t*>(K);
+    fw.q_mean = q_mean; fw.k_mean = k_mean; fw.index_out = index; fw.ctrl = ctrl; fw.inject = inject;
+    e = launch_kernel(attend_tc_k1_kernel<true>, dim3(grid), dim3(tc::THREADS), tc::SMEM_K1, st, false,
+                      maps, static_cast<const int32_t*>(index), lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, ctrl, d,
+                      tiles, fw);
     count_launch();
     return e;
 }

@@ -25,7 +25,6 @@ WsLayout ws_layout(const Dims& d) {
     while (blocks > 1024 && blocks % 2 == 0) blocks /= 2;
     L.dw_blocks = blocks;
     L.dw_part = off;  off += align256(sizeof(float) * (size_t)blocks * d.C * 26);
-    L.sync = off;     off += align256(sizeof(int32_t) * 2 * (size_t)d.B);
     L.total = off;
     return L;
 }
@@ -192,11 +191,12 @@ bra_status bra_forward(const bra_problem* p, const void* Q, const void* K, const
     int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
     float* qm = reinterpret_cast<float*>(w + L.q_mean);
     float* km = reinterpret_cast<float*>(w + L.k_mean);
-    // pooling, routing and attention in one launch, on request
-    if (p->impl == BRA_IMPL_TC_FUSED) {
-        if (!forward_tc_supported(d, p->dtype)) return BRA_ERR_UNSUPPORTED;
-        const cudaError_t e = launch_forward_tc(d, Q, K, V, lce_w, lce_b, O, idx, lse, qm, km, status,
-                                                reinterpret_cast<int32_t*>(w + L.sync), p->inject, st);
+    // pooling, routing and attention in one launch
+    static const bool one_launch = getenv("BRA_ONE_LAUNCH") != nullptr;     // tuning aid: also under BRA_IMPL_AUTO
+    if (p->impl == BRA_IMPL_TC_FUSED && !forward_tc_supported(d, p->dtype)) return BRA_ERR_UNSUPPORTED;
+    if (p->impl == BRA_IMPL_TC_FUSED ||
+        (one_launch && p->impl == BRA_IMPL_AUTO && path == PATH_TC && forward_tc_supported(d, p->dtype))) {
+        const cudaError_t e = launch_forward_tc(d, Q, K, V, lce_w, lce_b, O, idx, lse, qm, km, status, p->inject, st);
         return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;
     }
     s = run_route(d, p->dtype, Q, K, qm, km, idx, st);
@@ -237,26 +237,22 @@ bra_status bra_workspace_init(const bra_problem* p, void* ws, size_t ws_bytes, v
     if ((s = check_ws(d, ws, ws_bytes, &L)) != BRA_OK) return s;
     char* w = static_cast<char*>(ws);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the status block and the counters / flags of the one-launch forward; the rest is written before it is read
+    // the status block (error words, barrier counters of the one-launch forward); the rest is written before it is read
     if (cudaMemsetAsync(w + L.status, 0, 256, st) != cudaSuccess) return BRA_ERR_CUDA;
-    if (cudaMemsetAsync(w + L.sync, 0, L.total - L.sync, st) != cudaSuccess) return BRA_ERR_CUDA;
     return BRA_OK;
 }
 
 bra_status bra_device_status(void* ws, void* stream) {
     if (!ws) return BRA_ERR_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int32_t host[4] = {0, 0, 0, 0};     // code, detail; offset and size of the one-launch forward's counters
+    int32_t host[2] = {0, 0};           // code, detail
     if (cudaMemcpyAsync(host, ws, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return BRA_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return BRA_ERR_CUDA;
     if (host[0] != 0) {
-        // a kernel that gave up leaves its job counter, per-image counters and flags as they were: clear
-        // them with the error, so that the next call on this ws starts clean
+        // a kernel that gave up leaves its barrier counters as they were: clear the whole status block with
+        // the error, so that the next call on this ws starts clean
         if (cudaMemsetAsync(ws, 0, 256, st) != cudaSuccess) return BRA_ERR_CUDA;
-        if (host[2] >= 256 && host[3] > 0 &&
-            cudaMemsetAsync(static_cast<char*>(ws) + host[2], 0, (size_t)host[3], st) != cudaSuccess)
-            return BRA_ERR_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return BRA_ERR_CUDA;
     }
     if (host[0] < 0 || host[0] > BRA_ERR_TIMEOUT) return BRA_ERR_CUDA;

@@ -37,7 +37,6 @@ struct WsLayout {
     size_t inv_off;     // int32 [B,heads_i,R+1] CSR offsets of the inverse routing index
     size_t inv_list;    // int32 [B,heads_i,R*topk] query regions routed to each key region
     size_t dw_part;     // fp32 [dw_blocks, C*26] partial LCE weight / bias gradients
-    size_t sync;        // int32 [2,B] one-launch forward: pooled units per image, "image routed" flags (zero between calls)
     size_t total;
     int dw_blocks;
 };
@@ -80,8 +79,7 @@ cudaError_t launch_attend_tc(const Dims& d, const void* Q, const void* K, const 
 bool forward_tc_supported(const Dims& d, int dtype);
 cudaError_t launch_forward_tc(const Dims& d, const void* Q, const void* K, const void* V,
                               const float* lce_w, const float* lce_b, void* O, int32_t* index, float* lse,
-                              float* q_mean, float* k_mean, int32_t* ctrl, int32_t* sync, int inject,
-                              cudaStream_t st);
+                              float* q_mean, float* k_mean, int32_t* ctrl, int inject, cudaStream_t st);
 
 bool attend_img_supported(const Dims& d, int dtype);
 cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,

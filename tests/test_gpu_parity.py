@@ -439,7 +439,7 @@ def test_forward_orders_attention_after_routing(bra, n):
 
 
 # bf16, head dim 32, 8 x 8-token regions, topk = 1, per-head routing, <= 64 regions, C <= 128: with
-# BRA_IMPL_TC_FUSED bra_forward is ONE kernel launch (pooling, routing and attention as numbered jobs of one grid)
+# BRA_IMPL_TC_FUSED bra_forward is ONE launch (pooling, routing, attention: three phases of one grid)
 FUSED = 5
 ONE_LAUNCH_CASES = [
     BraConfig("fused-single-region", 1, 8, 8, 64, 2, 1, 1, "bf16"),
@@ -453,9 +453,9 @@ ONE_LAUNCH_CASES = [
 
 @pytest.mark.parametrize("cfg", ONE_LAUNCH_CASES, ids=[c.name for c in ONE_LAUNCH_CASES])
 def test_forward_in_one_launch_equals_route_then_attend(bra, cfg):
-    """The one-launch forward gives, bit for bit, the index of bra_route, and the O / lse of bra_attend up
-    to the rounding of a different summation order (it is another kernel), call after call on the same
-    scratch buffer (its counters and flags clean themselves); both match the oracle."""
+    """The one-launch forward gives, bit for bit, the index of bra_route and the O / lse of bra_attend,
+    call after call on the same scratch buffer (its barrier counters clean themselves), and matches
+    the oracle."""
     import torch
     p = problem_of(bra, cfg, impl=FUSED)
     ws = bra.workspace(p)
@@ -465,19 +465,13 @@ def test_forward_in_one_launch_equals_route_then_attend(bra, cfg):
         _, _, idx = bra.bra_route(p, t["Q"], t["K"], ws=ws)
         O, lse = bra.bra_attend(p, t["Q"], t["K"], t["V"], idx, t["w"], ws=ws)
         want.append((idx.clone(), O.clone(), lse.clone()))
-    seen = []
     for it in range(5):
         t, (idx_ref, O_ref, lse_ref) = sets[it % 2], want[it % 2]
         O, idx, lse = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
         assert bra.last_launch_count() == 1
         assert bra.bra_device_status(ws) == 0, f"call {it}"
         assert (idx == idx_ref).all(), f"call {it}"
-        assert (O.float() - O_ref.float()).abs().max().item() <= 2 ** -6, f"call {it}"     # a bf16 ulp at |O| < 4
-        assert (lse - lse_ref).abs().max().item() <= 1e-5, f"call {it}"
-        if it >= 2:
-            assert (O == seen[it % 2][0]).all() and (lse == seen[it % 2][1]).all(), f"call {it} differs from call {it - 2}"
-        else:
-            seen.append((O.clone(), lse.clone()))
+        assert (O == O_ref).all() and (lse == lse_ref).all(), f"call {it}"
     x = synthetic.make_inputs(cfg, seed=300)
     _, _, idx_o, gap = orc.bra_route(x["Q"], x["K"], cfg.heads, cfg.S, cfg.topk)
     check_index(want[0][0].cpu().numpy(), idx_o, gap, cfg.topk, cfg.R, oracle_affinity(x, cfg))
@@ -486,10 +480,10 @@ def test_forward_in_one_launch_equals_route_then_attend(bra, cfg):
 
 
 def test_bounded_wait_that_runs_out_is_reported_and_recoverable(bra):
-    """Failure detection without a GPU fault: with the injection switch the routing step of the
-    one-launch forward never raises its per-image flags, so the attention jobs' bounded waits run
-    out (nothing is in flight on the tensor cores at that point), the kernel returns, and the status
-    reads BRA_ERR_TIMEOUT.  Reading the status restores the scratch buffer: the next call is clean."""
+    """Failure detection without a GPU fault: with the injection switch one pooled unit of the
+    one-launch forward is never counted as done, so every CTA's bounded wait for the end of pooling runs
+    out (no tile copy and no tensor-core work has been issued at that point), the kernel returns, and the
+    status reads BRA_ERR_TIMEOUT.  Reading the status restores the scratch buffer: the next call is clean."""
     cfg = BraConfig("timeout", 3, 32, 32, 64, 2, 4, 1, "bf16")
     t = to_dev(synthetic.make_inputs(cfg, seed=9), cfg)
     p = problem_of(bra, cfg, impl=FUSED)
