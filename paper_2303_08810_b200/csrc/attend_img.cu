@@ -22,8 +22,7 @@ namespace bra {
 using namespace ptx;
 
 namespace img {
-constexpr int MAX_WARPS = 8;      // per CTA when two CTAs share an SM
-constexpr int MAX_WARPS_BIG = 16; // per CTA when a CTA has the SM to itself (large slices)
+constexpr int MAX_WARPS = 8;
 }  // namespace img
 
 struct ImgGeom {
@@ -33,103 +32,13 @@ struct ImgGeom {
     int nblocks;            // key blocks per unit = ceil(topk * n_r / 64)
     uint32_t mul_nr, mul_ws, mul_s, mul_tpr;
     int off_k, off_v, off_idx, off_w, off_st, smem_bytes;
-    int off_route;          // in-kernel routing only: Q^r, K^r (fp32, [R][33]) and the affinity rows (score bits, [R][R])
 };
 
-// order-preserving bits of an fp32 score (-0 and +0 tie), as in the stand-alone routing kernels
-__device__ __forceinline__ uint32_t img_score_bits(float s) {
-    s += 0.0f;
-    const uint32_t u = __float_as_uint(s);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
-// Routing of one (image, head) inside the attention kernel (the forward pass in one launch): region means
-// of the head's 32 channels of Q (from global memory) and K (from the resident slice), Eq. 4, Eq. 5.  Every
-// sum runs in the order of the stand-alone kernels (per column the token rows top to bottom, then the
-// columns left to right; the affinity over the channels in increasing order; score descending, lower region
-// first), so the index equals bra_route's bit for bit.  Writes the index rows to global memory and, as
-// token ids of the routed regions' first tokens, to s_idx.
-__device__ __noinline__ void img_route(uint32_t kbase, const uint8_t* Qb, uint8_t* scratch, int32_t* s_idx,
-                                       int32_t* index_rows, const Dims& dm, uint32_t mul_s, int tid, int nthreads) {
-    float* qr = reinterpret_cast<float*>(scratch);
-    float* kr = qr + dm.R * 33;
-    uint32_t* sc = reinterpret_cast<uint32_t*>(kr + dm.R * 33);
-    const size_t tok_bytes = (size_t)dm.C * 2, row_bytes = (size_t)dm.W * tok_bytes;
-    const float inv = 1.0f / (float)dm.n_r;
-    for (int item = tid; item < 2 * dm.R * 16; item += nthreads) {
-        const int cp = item & 15, rr = item >> 4;
-        const int tsr = rr >= dm.R, r = tsr ? rr - dm.R : rr;
-        const int ry = fdiv(r, dm.S, mul_s), rx = r - ry * dm.S;
-        // tokens in the order of the sums (columns left to right, inside a column top to bottom), sixteen
-        // loads in flight at a time
-        float sx = 0.f, sy = 0.f, ax = 0.f, ay = 0.f;
-        int x = 0, y = 0;
-        for (int base = 0; base < dm.n_r; base += 16) {
-            uint32_t w[16];
-            int lx = x, ly = y;
-#pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                w[u] = 0u;
-                if (base + u < dm.n_r) {
-                    const int ty = ry * dm.hs + ly, tx = rx * dm.ws + lx;
-                    if (tsr) {
-                        const int tok = ty * dm.W + tx;
-                        w[u] = lds_u32(kbase + tok * 64 + (((cp >> 2) ^ ((tok >> 1) & 3)) << 4) + (cp & 3) * 4);
-                    } else {
-                        w[u] = ldg_u32(Qb + (size_t)ty * row_bytes + (size_t)tx * tok_bytes + cp * 4);
-                    }
-                    if (++ly == dm.hs) { ly = 0; ++lx; }
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                if (base + u < dm.n_r) {
-                    ax += __uint_as_float(w[u] << 16);
-                    ay += __uint_as_float(w[u] & 0xffff0000u);
-                    if (++y == dm.hs) { y = 0; ++x; sx += ax; sy += ay; ax = 0.f; ay = 0.f; }
-                }
-            }
-        }
-        float* dst = (tsr ? kr : qr) + r * 33 + 2 * cp;
-        dst[0] = sx * inv;
-        dst[1] = sy * inv;
-    }
-    __syncthreads();
-    for (int item = tid; item < dm.R * 4; item += nthreads) {
-        const int i = item >> 2;
-        for (int j = item & 3; j < dm.R; j += 4) {
-            float acc = 0.f;
-#pragma unroll
-            for (int c = 0; c < 32; ++c) acc = fmaf(qr[i * 33 + c], kr[j * 33 + c], acc);
-            sc[i * dm.R + j] = img_score_bits(acc);
-        }
-    }
-    __syncthreads();
-    for (int item = tid; item < dm.R * dm.R; item += nthreads) {
-        const int i = item / dm.R, j = item - i * dm.R;
-        const uint32_t mine = sc[item];
-        const uint32_t* row = sc + i * dm.R;
-        int rank = 0;
-        for (int jj = 0; jj < dm.R; ++jj) {
-            const uint32_t other = row[jj];
-            rank += (other > mine) || (other == mine && jj < j);
-        }
-        if (rank < dm.topk) {
-            const int qy = fdiv(j, dm.S, mul_s), qx = j - qy * dm.S;
-            s_idx[i * dm.topk + rank] = qy * dm.hs * dm.W + qx * dm.ws;
-            index_rows[i * dm.topk + rank] = j;
-        }
-    }
-}
-
-// VAR: 0 = CTAs of up to 8 warps, two per SM (128 registers per thread); 1 = up to 5 warps, two per SM: room
-// for ~200 registers per thread; 2 = up to 16 warps, one per SM (128 registers): for slices so large that
-// only one CTA fits an SM anyway, twice the warps per SM.
-// ROUTE: the routing index is computed here (and written to `index_out`) instead of read from `index`.
-template <int VAR, int SHAPE, bool ROUTE>
-__global__ void __launch_bounds__(VAR == 1 ? 160 : VAR == 2 ? img::MAX_WARPS_BIG * 32 : img::MAX_WARPS * 32, VAR == 2 ? 1 : 2)
+// SMALL: CTAs of up to 5 warps (two per SM by shared memory): room for ~200 registers per thread.
+template <bool SMALL, int SHAPE>
+__global__ void __launch_bounds__(SMALL ? 160 : img::MAX_WARPS * 32, 2)
 attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
-                  const __nv_bfloat16* __restrict__ Vg, const int32_t* index, int32_t* index_out,
+                  const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
                   const float* __restrict__ lce_w, const float* __restrict__ lce_b,
                   __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
                   int32_t* __restrict__ status, Dims dm, ImgGeom gm) {
@@ -153,15 +62,10 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
     cp_async_commit();
     // LCE weights of the head as [tap][channel pair] (read back conflict-free)
     if (dm.lce) img_load_weights(smem + gm.off_w, lce_w + (size_t)h * 32 * 25, false, tid, nthreads);
+    pdl_wait();          // the index may come from the routing kernel this launch overlaps
+    // routing rows of this (image, head): coherent loads, checked once, kept as token ids (-1: bad entry)
     int32_t* s_idx = reinterpret_cast<int32_t*>(smem + gm.off_idx);
-    if (ROUTE) {
-        cp_async_wait<0>();
-        __syncthreads();                 // the K slice is in shared memory
-        img_route(sbase + gm.off_k, Qb, smem + gm.off_route, s_idx,
-                  index_out + ((size_t)b * dm.heads + h) * dm.R * dm.topk, dm, gm.mul_s, tid, nthreads);
-    } else {
-        pdl_wait();          // the index may come from the routing kernel this launch overlaps
-        // routing rows of this (image, head): coherent loads, checked once, kept as token ids (-1: bad entry)
+    {
         const int hi = dm.heads_i == 1 ? 0 : h;
         const int32_t* ib = index + ((size_t)b * dm.heads_i + hi) * dm.R * dm.topk;
         for (int e = tid; e < dm.R * dm.topk; e += nthreads) {
@@ -376,7 +280,7 @@ attend_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
 }
 
 // ------------------------------------------------------------------ host side
-static ImgGeom img_geom(const Dims& d, int nw, bool route = false) {
+static ImgGeom img_geom(const Dims& d, int nw) {
     ImgGeom g;
     g.nw = nw;
     g.tpr = (d.n_r + 15) / 16;
@@ -389,8 +293,6 @@ static ImgGeom img_geom(const Dims& d, int nw, bool route = false) {
     g.off_st = off;  off += nw * 2048;
     g.off_w = off;   off += 25 * 16 * 8;
     g.off_idx = off; off += ((d.R * d.topk * 4 + 15) / 16) * 16;
-    g.off_route = 0;
-    if (route) { g.off_route = off; off += ((2 * d.R * 33 * 4 + d.R * d.R * 4 + 15) / 16) * 16; }
     g.smem_bytes = off;
     return g;
 }
@@ -411,18 +313,11 @@ bool attend_img_supported(const Dims& d, int dtype) {
     return img_geom(d, 1).smem_bytes <= 200 * 1024;
 }
 
-typedef void (*AttendImgKernel)(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*, const int32_t*, int32_t*,
+typedef void (*AttendImgKernel)(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*, const int32_t*,
                                 const float*, const float*, __nv_bfloat16*, float*, int32_t*, Dims, ImgGeom);
-template <int VAR, bool ROUTE>
-static AttendImgKernel img_kernel_v(int shape) {
-    return shape == 44 ? attend_img_kernel<VAR, 44, ROUTE> : shape == 22 ? attend_img_kernel<VAR, 22, ROUTE> : attend_img_kernel<VAR, 0, ROUTE>;
-}
-template <bool ROUTE>
-static AttendImgKernel img_kernel_r(int var, int shape) {
-    return var == 1 ? img_kernel_v<1, ROUTE>(shape) : var == 2 ? img_kernel_v<2, ROUTE>(shape) : img_kernel_v<0, ROUTE>(shape);
-}
-static AttendImgKernel img_kernel(int var, int shape, bool route) {
-    return route ? img_kernel_r<true>(var, shape) : img_kernel_r<false>(var, shape);
+static AttendImgKernel img_kernel(bool small, int shape) {
+    if (small) return shape == 44 ? attend_img_kernel<true, 44> : shape == 22 ? attend_img_kernel<true, 22> : attend_img_kernel<true, 0>;
+    return shape == 44 ? attend_img_kernel<false, 44> : shape == 22 ? attend_img_kernel<false, 22> : attend_img_kernel<false, 0>;
 }
 static cudaError_t img_occupancy(AttendImgKernel kernel, int nw, int smem_bytes, int* occ) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
@@ -430,80 +325,59 @@ static cudaError_t img_occupancy(AttendImgKernel kernel, int nw, int smem_bytes,
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, kernel, nw * 32, smem_bytes);
 }
 
-// route: the kernel computes the routing index itself and writes it to index_out (the forward pass in one launch)
-static cudaError_t launch_img(const Dims& d, const void* Q, const void* K, const void* V,
-                              const int32_t* index, int32_t* index_out, bool route, const float* lce_w, const float* lce_b,
+cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
+                              const int32_t* index, const float* lce_w, const float* lce_b,
                               void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel) {
-    // Warps per CTA and kernel variant (see the kernel's VAR): among
+    // Warps per CTA and register variant (SMALL: up to ~200 registers, CTAs of at most 5 warps): among
     // the choices that let every CTA of the grid be resident at once, the one with the most warps per
     // SM (the roomier variant on a tie); if none does, the most warps per SM.  Remembered per shape.
     const long long grid = (long long)d.B * d.heads;
     const int shape = img_region_shape(d);
     // the choice depends on the whole problem shape (kernel instantiation, shared-memory size) and on the device
-    struct Memo { long long grid; int dev, H, W, C, S, topk, lce, route, nw, var; };
-    static thread_local Memo memo = {0, -1, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    struct Memo { long long grid; int dev, H, W, C, S, topk, lce, nw; bool small; };
+    static thread_local Memo memo = {0, -1, 0, 0, 0, 0, 0, 0, 0, false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     int best_nw = 0;
-    int best_var = 0;
+    bool best_small = false;
     if (memo.nw && memo.grid == grid && memo.dev == dev && memo.H == d.H && memo.W == d.W && memo.C == d.C &&
-        memo.S == d.S && memo.topk == d.topk && memo.lce == d.lce && memo.route == (int)route) {
+        memo.S == d.S && memo.topk == d.topk && memo.lce == d.lce) {
         best_nw = memo.nw;
-        best_var = memo.var;
+        best_small = memo.small;
     } else {
         const int sms = img_sm_count();
         int best_warps = -1;
         bool best_fits = false;
-        for (int nw = img::MAX_WARPS_BIG; nw >= 1; --nw) {
-            const ImgGeom g = img_geom(d, nw, route);
+        for (int nw = img::MAX_WARPS; nw >= 1; --nw) {
+            const ImgGeom g = img_geom(d, nw);
             if (g.smem_bytes > 200 * 1024) continue;
-            for (int var = 0; var <= 2; ++var) {
-                if ((var == 0 && nw > img::MAX_WARPS) || (var == 1 && nw > 5) || (var == 2 && nw <= img::MAX_WARPS)) continue;
+            for (int small = 0; small <= (nw <= 5 ? 1 : 0); ++small) {
                 int occ = 0;
-                const cudaError_t e = img_occupancy(img_kernel(var, shape, route), nw, g.smem_bytes, &occ);
+                const cudaError_t e = img_occupancy(img_kernel(small != 0, shape), nw, g.smem_bytes, &occ);
                 if (e != cudaSuccess) return e;
                 if (occ <= 0) continue;
                 const bool fits = (long long)occ * sms >= grid;
                 const int warps = occ * nw;
                 if ((fits && !best_fits) || (fits == best_fits && warps >= best_warps)) {
-                    best_fits = fits; best_warps = warps; best_nw = nw; best_var = var;
+                    best_fits = fits; best_warps = warps; best_nw = nw; best_small = small != 0;
                 }
             }
         }
         if (!best_nw) return cudaErrorInvalidConfiguration;
-        memo = Memo{grid, dev, d.H, d.W, d.C, d.S, d.topk, d.lce, (int)route, best_nw, best_var};
+        memo = Memo{grid, dev, d.H, d.W, d.C, d.S, d.topk, d.lce, best_nw, best_small};
     }
-    const ImgGeom g = img_geom(d, best_nw, route);
+    const ImgGeom g = img_geom(d, best_nw);
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(Q);
     const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(K);
     const __nv_bfloat16* v = static_cast<const __nv_bfloat16*>(V);
     const bool pdl = after_own_kernel;
-    AttendImgKernel kernel = img_kernel(best_var, shape, route);
+    AttendImgKernel kernel = img_kernel(best_small, shape);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
     if (e != cudaSuccess) return e;
     e = launch_kernel(kernel, dim3((unsigned)grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st, pdl,
-                      q, k, v, index, index_out, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, g);
+                      q, k, v, index, lce_w, lce_b, static_cast<__nv_bfloat16*>(O), lse, status, d, g);
     count_launch();
     return e;
-}
-
-cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
-                              const int32_t* index, const float* lce_w, const float* lce_b,
-                              void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel) {
-    return launch_img(d, Q, K, V, index, nullptr, false, lce_w, lce_b, O, lse, status, st, after_own_kernel);
-}
-
-// The forward pass in one launch for small maps: per-head routing (a head's routing needs only the 32
-// channels its CTA holds) and few enough regions for the affinity rows to sit in shared memory.
-bool forward_img_supported(const Dims& d, int dtype) {
-    return attend_img_supported(d, dtype) && d.heads_i == d.heads && d.R <= 64 &&
-           img_geom(d, 1, true).smem_bytes <= 200 * 1024;
-}
-
-cudaError_t launch_forward_img(const Dims& d, const void* Q, const void* K, const void* V,
-                               const float* lce_w, const float* lce_b, void* O, int32_t* index, float* lse,
-                               int32_t* status, cudaStream_t st) {
-    return launch_img(d, Q, K, V, index, index, true, lce_w, lce_b, O, lse, status, st, false);
 }
 
 }  // namespace bra

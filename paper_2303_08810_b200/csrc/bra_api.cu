@@ -199,12 +199,6 @@ bra_status bra_forward(const bra_problem* p, const void* Q, const void* K, const
         const cudaError_t e = launch_forward_tc(d, Q, K, V, lce_w, lce_b, O, idx, lse, qm, km, status, p->inject, st);
         return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;
     }
-    // small maps: the image-resident kernel pools and routes its own (image, head)
-    static const bool img_route = getenv("BRA_IMG_ROUTE") != nullptr;       // tuning aid (slower than the chain at present)
-    if (path == PATH_IMG && img_route && forward_img_supported(d, p->dtype)) {
-        const cudaError_t e = launch_forward_img(d, Q, K, V, lce_w, lce_b, O, idx, lse, status, st);
-        return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;
-    }
     s = run_route(d, p->dtype, Q, K, qm, km, idx, st);
     if (s != BRA_OK) return s;
     return run_attend(path, d, p->dtype, Q, K, V, idx, lce_w, lce_b, O, lse, status, st, true);

@@ -85,11 +85,6 @@ bool attend_img_supported(const Dims& d, int dtype);
 cudaError_t launch_attend_img(const Dims& d, const void* Q, const void* K, const void* V,
                               const int32_t* index, const float* lce_w, const float* lce_b,
                               void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel);
-// Algorithm 1 in one launch for small maps (the image-resident kernel computes its own routing index)
-bool forward_img_supported(const Dims& d, int dtype);
-cudaError_t launch_forward_img(const Dims& d, const void* Q, const void* K, const void* V,
-                               const float* lce_w, const float* lce_b, void* O, int32_t* index, float* lse,
-                               int32_t* status, cudaStream_t st);
 bool attend_tc_wide_supported(const Dims& d, int dtype);
 cudaError_t launch_attend_tc_wide(const Dims& d, const void* Q, const void* K, const void* V,
                                   const int32_t* index, const float* lce_w, const float* lce_b,
