@@ -19,8 +19,13 @@
  *   - Q, K, V, O, dO, dQ, dK, dV: [B, H, W, C], element type p->dtype, channel
  *     c = head * (C / heads) + j (concat order of Eq. 2).
  *   - Regions: S x S non-overlapping blocks of (H/S) x (W/S) tokens, numbered
- *     row-major r = ry * S + rx (region partition, Section 3.2).  S must divide
- *     H and W.
+ *     row-major r = ry * S + rx (region partition, Section 3.2).  Where S does
+ *     not divide H or W (Appendix C picks S as a divisor "to avoid padding"),
+ *     the library works on copies of Q, K, V zero-padded at the bottom and the
+ *     right to the next multiples of S: the zero tokens are pooled, routed to
+ *     and attended to like real ones, and O, lse and the gradients are cropped
+ *     back to H x W.  The copies live in ws (bra_workspace_bytes accounts for
+ *     them) and cost one extra kernel per tensor.
  *   - index: int32 [B, heads, S*S, topk] (or [B, 1, S*S, topk] when
  *     p->shared_routing != 0).  Row i lists the key regions that the queries of
  *     region i attend to.  It is a list: any order, duplicates count twice.
@@ -50,7 +55,7 @@ extern "C" {
 typedef enum bra_status {
     BRA_OK = 0,
     BRA_ERR_NULL = 1,        /* a required pointer is NULL */
-    BRA_ERR_SHAPE = 2,       /* B,H,W,C,heads,S <= 0; S does not divide H or W; heads does not divide C */
+    BRA_ERR_SHAPE = 2,       /* B,H,W,C,heads,S <= 0; heads does not divide C */
     BRA_ERR_TOPK = 3,        /* topk < 1 or topk > S*S */
     BRA_ERR_DTYPE = 4,       /* dtype is not BRA_F32 / BRA_BF16 */
     BRA_ERR_ALIGN = 5,       /* a pointer is not 16-byte aligned (ws: 256) */
@@ -155,6 +160,8 @@ bra_status bra_route(const bra_problem* p, const void* Q, const void* K,
  *     them.  The array keeps the previous call's means; nothing in it has to
  *     be zero, because pooling overwrites every element routing then reads.
  *   - The region means are not returned; use bra_route to get them.
+ *   - S must divide H and W here (BRA_ERR_UNSUPPORTED otherwise): the padded
+ *     copies of Q and K that bra_route makes for other maps would need scratch.
  */
 #define BRA_ROUTE_STATIC_MAX_MEAN_FLOATS (512 * 1024)
 bra_status bra_route_static(const bra_problem* p, const void* Q, const void* K,

@@ -20,6 +20,11 @@ design notes of the repository):
   * top-k order: score descending, ties to the lower region index
   * LCE: 5x5 depthwise cross-correlation over the whole H x W map of V,
     stride 1, zero padding 2 (Section 3.2, Eq. 7)
+  * a map whose sides S does not divide (Appendix C only says that S is chosen
+    as a divisor "to avoid padding"): Q, K, V are zero-padded at the bottom and
+    right to the next multiples of S, the padded map is processed as any other
+    (the zero tokens are pooled, routed to and attended to like real ones),
+    and O, lse and the gradients are cropped back
 """
 from __future__ import annotations
 
@@ -167,6 +172,34 @@ def lce(V, w, bias=None):
 
 
 # ----------------------------------------------------------------------------
+# Maps that S does not divide (Appendix C): zero padding, then cropping
+# ----------------------------------------------------------------------------
+def padded_size(H, W, S):
+    """Next multiples of S."""
+    return -(-H // S) * S, -(-W // S) * S
+
+
+def pad_map(X, S):
+    """[B,H,W,C] -> [B,Hp,Wp,C]: zeros appended at the bottom and at the right."""
+    X = np.asarray(X, dtype=F64)
+    B, H, W, C = X.shape
+    Hp, Wp = padded_size(H, W, S)
+    out = np.zeros((B, Hp, Wp, C), dtype=F64)
+    out[:, :H, :W] = X
+    return out
+
+
+def crop_map(X, H, W):
+    """The top-left H x W tokens of a padded map."""
+    return np.ascontiguousarray(X[:, :H, :W])
+
+
+def _crop_lse(lse, Hp, Wp, H, W):
+    B, heads, _ = lse.shape
+    return np.ascontiguousarray(lse.reshape(B, heads, Hp, Wp)[:, :, :H, :W]).reshape(B, heads, H * W)
+
+
+# ----------------------------------------------------------------------------
 # The four calls of the boundary, on host arrays
 # ----------------------------------------------------------------------------
 def default_scale(C, heads):
@@ -175,6 +208,8 @@ def default_scale(C, heads):
 
 def bra_route(Q, K, heads, S, topk, shared_routing=False):
     """Q, K -> (Q^r, K^r [B,S^2,C], I^r int32 [B,heads|1,S^2,k], gap_rel)."""
+    if Q.shape[1] % S or Q.shape[2] % S:
+        Q, K = pad_map(Q, S), pad_map(K, S)
     Qr, Kr = region_means(Q, S), region_means(K, S)
     A = region_affinity(Qr, Kr, heads, shared_routing)
     index, gap = topk_index(A, topk)
@@ -183,6 +218,11 @@ def bra_route(Q, K, heads, S, topk, shared_routing=False):
 
 def bra_attend(Q, K, V, index, w, heads, S, scale=None, bias=None):
     """Eq. 7: O = Attention(Q, K^g, V^g) + LCE(V).  w=None disables LCE."""
+    H, W = Q.shape[1], Q.shape[2]
+    if H % S or W % S:
+        Hp, Wp = padded_size(H, W, S)
+        O, lse = bra_attend(pad_map(Q, S), pad_map(K, S), pad_map(V, S), index, w, heads, S, scale, bias)
+        return crop_map(O, H, W), _crop_lse(lse, Hp, Wp, H, W)
     C = Q.shape[-1]
     scale = default_scale(C, heads) if scale is None else scale
     O, lse = routed_attention(Q, K, V, index, heads, S, scale)
@@ -209,6 +249,10 @@ def bra_backward(Q, K, V, index, w, dO, heads, S, scale=None):
     w: dV += correlation-transpose(dO, w), dw[c,i,j] = sum dO[.,y,x,c] V[.,y+i-2,x+j-2,c].
     Returns dQ, dK, dV [B,H,W,C], dw [C,5,5], dbias [C].
     """
+    if np.shape(Q)[1] % S or np.shape(Q)[2] % S:
+        H0, W0 = np.shape(Q)[1], np.shape(Q)[2]
+        g = bra_backward(pad_map(Q, S), pad_map(K, S), pad_map(V, S), index, w, pad_map(dO, S), heads, S, scale)
+        return crop_map(g[0], H0, W0), crop_map(g[1], H0, W0), crop_map(g[2], H0, W0), g[3], g[4]
     Q = np.asarray(Q, dtype=F64)
     K = np.asarray(K, dtype=F64)
     V = np.asarray(V, dtype=F64)

@@ -25,6 +25,13 @@ WsLayout ws_layout(const Dims& d) {
     while (blocks > 1024 && blocks % 2 == 0) blocks /= 2;
     L.dw_blocks = blocks;
     L.dw_part = off;  off += align256(sizeof(float) * (size_t)blocks * d.C * 26);
+    L.pad = L.pad_lse = off;
+    L.pad_tensor = 0;
+    if (d.H != d.H0 || d.W != d.W0) {
+        L.pad_tensor = align256((size_t)d.B * d.N * d.C * d.esize);
+        L.pad = off;      off += 7 * L.pad_tensor;
+        L.pad_lse = off;  off += align256(sizeof(float) * (size_t)d.B * d.heads * d.N);
+    }
     L.total = off;
     return L;
 }
@@ -34,20 +41,24 @@ static bra_status make_dims(const bra_problem* p, Dims* out) {
     if (!p) return BRA_ERR_NULL;
     if (p->B <= 0 || p->H <= 0 || p->W <= 0 || p->C <= 0 || p->heads <= 0 || p->S <= 0)
         return BRA_ERR_SHAPE;
-    if (p->H % p->S || p->W % p->S || p->C % p->heads) return BRA_ERR_SHAPE;
-    if ((int64_t)p->B * p->H * p->W * p->C >= ((int64_t)1 << 40)) return BRA_ERR_SHAPE;
+    if (p->C % p->heads) return BRA_ERR_SHAPE;
+    // S need not divide H, W: the map is zero-padded at the bottom and right to the next multiples of S
+    const int Hp = (p->H + p->S - 1) / p->S * p->S, Wp = (p->W + p->S - 1) / p->S * p->S;
+    if ((int64_t)p->B * Hp * Wp * p->C >= ((int64_t)1 << 40)) return BRA_ERR_SHAPE;
     if (p->topk < 1 || (int64_t)p->topk > (int64_t)p->S * p->S) return BRA_ERR_TOPK;
     if (p->dtype != BRA_F32 && p->dtype != BRA_BF16) return BRA_ERR_DTYPE;
     if (p->lce_ksize != 0 && p->lce_ksize != 5) return BRA_ERR_UNSUPPORTED;
     if (p->impl < BRA_IMPL_AUTO || p->impl > BRA_IMPL_TC_FUSED) return BRA_ERR_UNSUPPORTED;
     if (p->inject != BRA_INJECT_NONE && p->inject != BRA_INJECT_HOLD_ROUTE_FLAGS) return BRA_ERR_UNSUPPORTED;
     Dims d;
-    d.B = p->B; d.H = p->H; d.W = p->W; d.C = p->C; d.heads = p->heads; d.S = p->S; d.topk = p->topk;
+    d.B = p->B; d.H = Hp; d.W = Wp; d.C = p->C; d.heads = p->heads; d.S = p->S; d.topk = p->topk;
+    d.H0 = p->H; d.W0 = p->W;
+    d.esize = p->dtype == BRA_BF16 ? 2 : 4;
     d.d = p->C / p->heads;
     d.R = p->S * p->S;
-    d.hs = p->H / p->S; d.ws = p->W / p->S;
+    d.hs = Hp / p->S; d.ws = Wp / p->S;
     d.n_r = d.hs * d.ws;
-    d.N = p->H * p->W;
+    d.N = Hp * Wp;
     d.heads_i = p->shared_routing ? 1 : p->heads;
     d.lce = p->lce_ksize == 5;
     d.scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)d.d);
@@ -70,6 +81,24 @@ static bra_status check_ws(const Dims& d, const void* ws, size_t ws_bytes, WsLay
     *L = ws_layout(d);
     if (ws_bytes < L->total) return BRA_ERR_WORKSPACE;
     return BRA_OK;
+}
+
+static bool padded(const Dims& d) { return d.H != d.H0 || d.W != d.W0; }
+
+// The zero-padded copy of a caller's map in slot `slot` of the scratch buffer (or the map itself if S divides it).
+static const void* pad_in(const Dims& d, const WsLayout& L, char* w, int slot, const void* src, cudaStream_t st, bool* ok) {
+    if (!padded(d)) return src;
+    void* dst = w + L.pad + slot * L.pad_tensor;
+    if (launch_pad_copy(src, dst, d.B, d.H0, d.W0, d.H, d.W, d.C * d.esize, true, st) != cudaSuccess) *ok = false;
+    return dst;
+}
+static void* pad_out(const Dims& d, const WsLayout& L, char* w, int slot, void* dst) {
+    return padded(d) ? static_cast<void*>(w + L.pad + slot * L.pad_tensor) : dst;
+}
+static void crop_out(const Dims& d, const WsLayout& L, char* w, int slot, void* dst, cudaStream_t st, bool* ok) {
+    if (!padded(d) || !dst) return;
+    if (launch_pad_copy(w + L.pad + slot * L.pad_tensor, dst, d.B, d.H0, d.W0, d.H, d.W, d.C * d.esize, false, st) != cudaSuccess)
+        *ok = false;
 }
 
 enum Path { PATH_NONE, PATH_SIMT, PATH_MMA, PATH_TC, PATH_TC_WIDE, PATH_IMG };
@@ -144,7 +173,12 @@ bra_status bra_route(const bra_problem* p, const void* Q, const void* K,
     char* w = static_cast<char*>(ws);
     float* qm = q_mean ? q_mean : reinterpret_cast<float*>(w + L.q_mean);
     float* km = k_mean ? k_mean : reinterpret_cast<float*>(w + L.k_mean);
-    return run_route(d, p->dtype, Q, K, qm, km, index, static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    bool ok = true;
+    Q = pad_in(d, L, w, 0, Q, st, &ok);
+    K = pad_in(d, L, w, 1, K, st, &ok);
+    if (!ok) return BRA_ERR_CUDA;
+    return run_route(d, p->dtype, Q, K, qm, km, index, st);
 }
 
 bra_status bra_attend(const bra_problem* p, const void* Q, const void* K, const void* V,
@@ -164,8 +198,20 @@ bra_status bra_attend(const bra_problem* p, const void* Q, const void* K, const 
     Path path = choose_attend(d, p->dtype, p->impl);
     if (path == PATH_NONE) return BRA_ERR_UNSUPPORTED;
     char* w = static_cast<char*>(ws);
-    return run_attend(path, d, p->dtype, Q, K, V, index, lce_w, lce_b, O, lse,
-                      reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(stream), false);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    bool ok = true;
+    Q = pad_in(d, L, w, 0, Q, st, &ok);
+    K = pad_in(d, L, w, 1, K, st, &ok);
+    V = pad_in(d, L, w, 2, V, st, &ok);
+    if (!ok) return BRA_ERR_CUDA;
+    float* lse_k = (lse && padded(d)) ? reinterpret_cast<float*>(w + L.pad_lse) : lse;
+    s = run_attend(path, d, p->dtype, Q, K, V, index, lce_w, lce_b, pad_out(d, L, w, 3, O), lse_k,
+                   reinterpret_cast<int32_t*>(w + L.status), st, false);
+    if (s != BRA_OK) return s;
+    crop_out(d, L, w, 3, O, st, &ok);
+    if (lse && padded(d) &&
+        launch_pad_copy(lse_k, lse, (long long)d.B * d.heads, d.H0, d.W0, d.H, d.W, 4, false, st) != cudaSuccess) ok = false;
+    return ok ? BRA_OK : BRA_ERR_CUDA;
 }
 
 bra_status bra_forward(const bra_problem* p, const void* Q, const void* K, const void* V,
@@ -191,17 +237,33 @@ bra_status bra_forward(const bra_problem* p, const void* Q, const void* K, const
     int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
     float* qm = reinterpret_cast<float*>(w + L.q_mean);
     float* km = reinterpret_cast<float*>(w + L.k_mean);
+    bool ok = true;
+    Q = pad_in(d, L, w, 0, Q, st, &ok);
+    K = pad_in(d, L, w, 1, K, st, &ok);
+    V = pad_in(d, L, w, 2, V, st, &ok);
+    if (!ok) return BRA_ERR_CUDA;
+    void* O_user = O;
+    float* lse_user = lse;
+    O = pad_out(d, L, w, 3, O);
+    if (lse && padded(d)) lse = reinterpret_cast<float*>(w + L.pad_lse);
+    auto finish = [&](bra_status rs) -> bra_status {
+        if (rs != BRA_OK) return rs;
+        crop_out(d, L, w, 3, O_user, st, &ok);
+        if (lse_user && padded(d) &&
+            launch_pad_copy(lse, lse_user, (long long)d.B * d.heads, d.H0, d.W0, d.H, d.W, 4, false, st) != cudaSuccess) ok = false;
+        return ok ? BRA_OK : BRA_ERR_CUDA;
+    };
     // pooling, routing and attention in one launch
     static const bool one_launch = getenv("BRA_ONE_LAUNCH") != nullptr;     // tuning aid: also under BRA_IMPL_AUTO
     if (p->impl == BRA_IMPL_TC_FUSED && !forward_tc_supported(d, p->dtype)) return BRA_ERR_UNSUPPORTED;
     if (p->impl == BRA_IMPL_TC_FUSED ||
         (one_launch && p->impl == BRA_IMPL_AUTO && path == PATH_TC && forward_tc_supported(d, p->dtype))) {
         const cudaError_t e = launch_forward_tc(d, Q, K, V, lce_w, lce_b, O, idx, lse, qm, km, status, p->inject, st);
-        return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;
+        return finish(e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA);
     }
     s = run_route(d, p->dtype, Q, K, qm, km, idx, st);
     if (s != BRA_OK) return s;
-    return run_attend(path, d, p->dtype, Q, K, V, idx, lce_w, lce_b, O, lse, status, st, true);
+    return finish(run_attend(path, d, p->dtype, Q, K, V, idx, lce_w, lce_b, O, lse, status, st, true));
 }
 
 bra_status bra_backward(const bra_problem* p, const void* Q, const void* K, const void* V,
@@ -222,10 +284,26 @@ bra_status bra_backward(const bra_problem* p, const void* Q, const void* K, cons
     WsLayout L;
     if ((s = check_ws(d, ws, ws_bytes, &L)) != BRA_OK) return s;
     if (!backward_supported(d)) return BRA_ERR_UNSUPPORTED;
-    cudaError_t e = launch_backward(d, p->dtype, p->impl, Q, K, V, index, lce_w, lse, dO, dQ, dK, dV,
-                                    d_lce_w, d_lce_b, static_cast<char*>(ws), L,
-                                    static_cast<cudaStream_t>(stream));
-    return e == cudaSuccess ? BRA_OK : BRA_ERR_CUDA;
+    char* w = static_cast<char*>(ws);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    bool ok = true;
+    Q = pad_in(d, L, w, 0, Q, st, &ok);
+    K = pad_in(d, L, w, 1, K, st, &ok);
+    V = pad_in(d, L, w, 2, V, st, &ok);
+    dO = pad_in(d, L, w, 3, dO, st, &ok);          // zero in the padding: padded queries contribute nothing
+    if (padded(d)) {                               // lse of the padded queries: 0 (their scores are 0, their P finite)
+        float* lp = reinterpret_cast<float*>(w + L.pad_lse);
+        if (launch_pad_copy(lse, lp, (long long)d.B * d.heads, d.H0, d.W0, d.H, d.W, 4, true, st) != cudaSuccess) ok = false;
+        lse = lp;
+    }
+    if (!ok) return BRA_ERR_CUDA;
+    cudaError_t e = launch_backward(d, p->dtype, p->impl, Q, K, V, index, lce_w, lse, dO, pad_out(d, L, w, 4, dQ),
+                                    pad_out(d, L, w, 5, dK), pad_out(d, L, w, 6, dV), d_lce_w, d_lce_b, w, L, st);
+    if (e != cudaSuccess) return BRA_ERR_CUDA;
+    crop_out(d, L, w, 4, dQ, st, &ok);
+    crop_out(d, L, w, 5, dK, st, &ok);
+    crop_out(d, L, w, 6, dV, st, &ok);
+    return ok ? BRA_OK : BRA_ERR_CUDA;
 }
 
 bra_status bra_workspace_init(const bra_problem* p, void* ws, size_t ws_bytes, void* stream) {

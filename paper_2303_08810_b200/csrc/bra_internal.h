@@ -25,6 +25,10 @@ struct Dims {
     int heads_i;  // heads of the routing index: heads, or 1 with shared routing
     int lce;      // 1: add LCE
     float scale;  // softmax scale (Eq. 1)
+    // When S does not divide the caller's map, H and W above are the padded sizes (next multiples of S: the
+    // kernels only ever see a divisible map) and these are the caller's; equal to H, W otherwise.
+    int H0, W0;
+    int esize;    // bytes per element of Q, K, V, O
 };
 
 // Scratch layout (byte offsets from ws, all multiples of 256).
@@ -37,6 +41,9 @@ struct WsLayout {
     size_t inv_off;     // int32 [B,heads_i,R+1] CSR offsets of the inverse routing index
     size_t inv_list;    // int32 [B,heads_i,R*topk] query regions routed to each key region
     size_t dw_part;     // fp32 [dw_blocks, C*26] partial LCE weight / bias gradients
+    size_t pad;         // padded maps only: seven [B,H,W,C] tensors of the padded size (Q, K, V, O / dO, dQ, dK, dV)
+    size_t pad_lse;     // padded maps only: fp32 [B,heads,H*W] of the padded size
+    size_t pad_tensor;  // bytes of one padded tensor
     size_t total;
     int dw_blocks;
 };
@@ -51,6 +58,10 @@ void reset_launch_count();
 bra_status check_problem(const bra_problem* p, Dims* out);
 
 // ---- kernel launchers (each returns the cudaError of its launches) ----------
+// Copies between the caller's [B,H0,W0,C] map and the zero-padded [B,H,W,C] map the kernels work on
+// (to_padded: fill; else crop).  elem_bytes: bytes of one token (C * element size; a multiple of 4).
+cudaError_t launch_pad_copy(const void* src, void* dst, long long images, int H0, int W0, int H, int W,
+                            int token_bytes, bool to_padded, cudaStream_t st);
 cudaError_t launch_pool(const Dims& d, int dtype, const void* Q, const void* K,
                         float* q_mean, float* k_mean, cudaStream_t st);
 cudaError_t launch_route(const Dims& d, const float* q_mean, const float* k_mean,

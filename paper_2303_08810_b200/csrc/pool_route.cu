@@ -541,4 +541,48 @@ cudaError_t launch_route(const Dims& d, const float* q_mean, const float* k_mean
     return launch_route_e<8>(d, q_mean, k_mean, index, st);
 }
 
+// ------------------------------------------------------------------ maps that S does not divide
+// The kernels work on maps whose sides are multiples of S; a caller's map of another size is copied into a
+// zero-padded one (padding at the bottom and right) and the results are cropped back.  T: uint4 when a
+// token's bytes are a multiple of 16, else uint32_t.
+template <typename T>
+__global__ void __launch_bounds__(256)
+pad_copy_kernel(const T* __restrict__ src, T* __restrict__ dst, long long images, int H0, int W0, int H, int W,
+                int tvec, bool to_padded) {
+    const int Ho = to_padded ? H : H0, Wo = to_padded ? W : W0;        // the map that is written
+    const long long total = images * Ho * Wo * tvec;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+        const int v = (int)(e % tvec);
+        long long t = e / tvec;
+        const int x = (int)(t % Wo); t /= Wo;
+        const int y = (int)(t % Ho);
+        const long long b = t / Ho;
+        T val = T();
+        if (to_padded) {
+            if (y < H0 && x < W0) val = src[((b * H0 + y) * W0 + x) * tvec + v];
+        } else {
+            val = src[((b * H + y) * W + x) * tvec + v];
+        }
+        dst[e] = val;
+    }
+}
+
+cudaError_t launch_pad_copy(const void* src, void* dst, long long images, int H0, int W0, int H, int W,
+                            int token_bytes, bool to_padded, cudaStream_t st) {
+    const bool wide = token_bytes % 16 == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0;
+    const int tvec = token_bytes / (wide ? 16 : 4);
+    const long long total = images * (to_padded ? (long long)H * W : (long long)H0 * W0) * tvec;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks < 1) blocks = 1;
+    if (wide)
+        pad_copy_kernel<uint4><<<(unsigned)blocks, 256, 0, st>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst),
+                                                                 images, H0, W0, H, W, tvec, to_padded);
+    else
+        pad_copy_kernel<uint32_t><<<(unsigned)blocks, 256, 0, st>>>(static_cast<const uint32_t*>(src), static_cast<uint32_t*>(dst),
+                                                                    images, H0, W0, H, W, tvec, to_padded);
+    count_launch();
+    return cudaGetLastError();
+}
+
 }  // namespace bra

@@ -50,6 +50,7 @@ extern "C" bra_status bra_route_static(const bra_problem* p, const void* Q, cons
     const size_t mean_floats = (size_t)d.B * d.R * d.C;
     if (mean_floats > (size_t)BRA_ROUTE_STATIC_MAX_MEAN_FLOATS) return BRA_ERR_STATIC_LIMIT;
     if (!route_supported(d)) return BRA_ERR_UNSUPPORTED;
+    if (d.H != d.H0 || d.W != d.W0) return BRA_ERR_UNSUPPORTED;      // a padded copy of Q and K would need scratch
     float* means = nullptr;
     if ((s = means_address(&means)) != BRA_OK) return s;
     float* q_mean = means;

@@ -60,14 +60,15 @@ def test_workspace_bytes(lib):
     # holds at least the two mean tensors and the index
     assert n >= 2 * 4 * p.B * 16 * p.C + 4 * p.B * p.heads * 16 * p.topk
     assert binding.workspace_bytes(problem(B=4)) > n
-    assert binding.workspace_bytes(problem(S=3)) == 0          # invalid problem
+    assert binding.workspace_bytes(problem(S=0)) == 0          # invalid problem
+    assert binding.workspace_bytes(problem(S=3)) > n           # S does not divide the map: room for the padded copies
 
 
 A = 0x10000  # a fake, aligned, never dereferenced device address
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(B=0), 2), (dict(H=-1), 2), (dict(S=3), 2), (dict(S=0), 2), (dict(heads=3), 2),
+    (dict(B=0), 2), (dict(H=-1), 2), (dict(S=0), 2), (dict(heads=3), 2),
     (dict(topk=0), 3), (dict(topk=17), 3),
 ])
 def test_route_rejects_bad_problems(lib, kw, code):

@@ -520,6 +520,49 @@ def test_workspace_init_makes_a_dirty_buffer_usable(bra):
     assert (O == O_ref).all() and (idx == idx_ref).all()
 
 
+# ------------------------------------------------------------------ maps S does not divide (Appendix C)
+PADDED_CASES = [
+    BraConfig("pad-8x8-regions-k1", 2, 30, 29, 64, 2, 4, 1, "bf16"),          # padded to 32 x 32: tcgen05, topk = 1
+    BraConfig("pad-8x8-regions-k3", 1, 61, 63, 64, 2, 8, 3, "bf16"),          # padded to 64 x 64: tcgen05, any topk
+    BraConfig("pad-small-map-many-images", 40, 13, 13, 64, 2, 7, 4, "bf16"),  # padded to 14 x 14: image-resident
+    BraConfig("pad-small-map", 3, 13, 14, 64, 2, 7, 4, "bf16"),               # warp-level kernel
+    BraConfig("pad-wide-regions", 1, 30, 31, 64, 2, 2, 2, "bf16"),            # padded to 32 x 32, 16 x 16 regions
+    BraConfig("pad-fp32", 1, 15, 14, 32, 1, 4, 2, "f32"),
+]
+
+
+@pytest.mark.parametrize("cfg", PADDED_CASES, ids=[c.name for c in PADDED_CASES])
+def test_maps_that_S_does_not_divide(bra, cfg):
+    """Forward and backward on a map zero-padded (inside the library) to the next multiples of S, against
+    the oracle's padded reading: index of the padded map's regions, O / lse / gradients of the caller's size."""
+    x = synthetic.make_inputs(cfg, seed=77, with_do=True)
+    t = to_dev(x, cfg)
+    p = problem_of(bra, cfg)
+    ws = bra.workspace(p)
+    O, idx, lse = bra.bra_forward(p, t["Q"], t["K"], t["V"], t["w"], ws=ws)
+    assert bra.bra_device_status(ws) == 0
+    assert tuple(O.shape) == (cfg.B, cfg.H, cfg.W, cfg.C) and tuple(lse.shape) == (cfg.B, cfg.heads, cfg.H * cfg.W)
+    Qr, Kr, idx_ref, gap = orc.bra_route(x["Q"], x["K"], cfg.heads, cfg.S, cfg.topk)
+    A = orc.region_affinity(Qr, Kr, cfg.heads)
+    check_index(idx.cpu().numpy(), idx_ref, gap, cfg.topk, cfg.R, A)
+    idn = idx.cpu().numpy()
+    O_ref, lse_ref = orc.bra_attend(x["Q"], x["K"], x["V"], idn, x["w"], cfg.heads, cfg.S)
+    check_O(f64(O), O_ref, cfg.dtype)
+    np.testing.assert_allclose(f64(lse), lse_ref, rtol=0, atol=1e-5 if cfg.dtype == "f32" else 2e-3)
+    # the two-call form gives the same
+    qm, km, idx2 = bra.bra_route(p, t["Q"], t["K"], ws=ws)
+    O2, lse2 = bra.bra_attend(p, t["Q"], t["K"], t["V"], idx2, t["w"], ws=ws)
+    assert (idx2 == idx).all() and (O2 == O).all()
+    np.testing.assert_allclose(f64(qm), Qr, rtol=0, atol=2e-6)
+    g = bra.bra_backward(p, t["Q"], t["K"], t["V"], idx, t["w"], lse, t["dO"], ws=ws, want_bias_grad=True)
+    assert bra.bra_device_status(ws) == 0
+    ref = orc.bra_backward(x["Q"], x["K"], x["V"], idn, x["w"], x["dO"], cfg.heads, cfg.S)
+    tol = GRAD_MAX if cfg.dtype == "bf16" else 2e-4
+    for name, a, r in zip(("dQ", "dK", "dV", "d_lce_w", "d_lce_b"), g, ref):
+        assert tuple(a.shape) == r.shape, name
+        assert np.abs(f64(a) - r).max() <= tol, f"{cfg.name} {name}"
+
+
 # ------------------------------------------------------------------ backward
 def run_backward_case(bra, cfg, seed, clustered=False, shared=False, index=None, impl="auto"):
     import torch

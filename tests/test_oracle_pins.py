@@ -448,6 +448,89 @@ def test_backward_full_attention_case_matches_textbook_gradient():
         np.testing.assert_allclose(ours, ref, rtol=1e-10, atol=1e-12)
 
 
+# ---------------------------------------------------------------- maps S does not divide (Appendix C)
+def hand_padded(X, S):
+    """Zero padding at the bottom and right, token by token (not the oracle's slicing)."""
+    B, H, W, C = X.shape
+    Hp, Wp = math.ceil(H / S) * S, math.ceil(W / S) * S
+    out = np.zeros((B, Hp, Wp, C))
+    for b, y, x in itertools.product(range(B), range(H), range(W)):
+        out[b, y, x] = X[b, y, x]
+    return out
+
+
+def test_pad_and_crop_place_every_token_by_hand():
+    X = rng(40).standard_normal((2, 5, 7, 3))
+    P = orc.pad_map(X, 3)
+    assert P.shape == (2, 6, 9, 3) and orc.padded_size(5, 7, 3) == (6, 9)
+    np.testing.assert_array_equal(P, hand_padded(X, 3))
+    np.testing.assert_array_equal(orc.crop_map(P, 5, 7), X)
+    Y = rng(41).standard_normal((1, 6, 9, 3))
+    np.testing.assert_array_equal(orc.pad_map(Y, 3), Y)          # a map S divides is left alone
+
+
+def test_padded_map_with_all_regions_is_full_attention_over_real_and_zero_tokens():
+    """topk = S^2 on a 5 x 7 map with S = 2: every query attends to all 6 x 8 tokens of the padded map,
+    the 18 zero tokens included (score 0, value 0); O and lse of the real queries equal the textbook
+    routine run on hand-padded arrays, and the LCE term is the correlation of the UNPADDED V."""
+    from scipy.signal import correlate2d
+    B, H, W, C, heads, S = 1, 5, 7, 4, 2, 2
+    g = rng(42)
+    Q, K, V = (g.standard_normal((B, H, W, C)) for _ in range(3))
+    w = g.standard_normal((C, 5, 5))
+    scale = 0.41
+    O, index, lse, _ = orc.bra_forward(Q, K, V, w, heads, S, S * S, scale=scale)
+    assert O.shape == Q.shape and lse.shape == (B, heads, H * W) and index.shape == (B, heads, S * S, S * S)
+    Of, lsef = full_attention_loops(hand_padded(Q, S), hand_padded(K, S), hand_padded(V, S), heads, scale)
+    conv = np.stack([correlate2d(V[0, :, :, c], w[c], mode="same", boundary="fill", fillvalue=0.0)
+                     for c in range(C)], axis=-1)[None]
+    np.testing.assert_allclose(O, Of[:, :H, :W] + conv, rtol=1e-11, atol=1e-12)
+    lse_ref = lsef.reshape(B, heads, 6, 8)[:, :, :H, :W].reshape(B, heads, H * W)
+    np.testing.assert_allclose(lse, lse_ref, rtol=1e-11, atol=1e-12)
+
+
+def test_padded_routing_pools_the_zero_tokens_and_matches_the_whole_map_scan():
+    """Region means of a padded map divide by the full region size (zeros count); routed attention on
+    the padded map equals the per-query scan over hand-padded arrays."""
+    B, H, W, C, heads, S, k = 1, 5, 5, 4, 2, 3, 2
+    g = rng(43)
+    Q, K, V = (g.standard_normal((B, H, W, C)) for _ in range(3))
+    Qr, Kr, index, _ = orc.bra_route(Q, K, heads, S, k)
+    Kp = hand_padded(K, S)
+    for r in range(S * S):
+        ry, rx = divmod(r, S)
+        np.testing.assert_allclose(Kr[0, r], Kp[0, 2 * ry:2 * ry + 2, 2 * rx:2 * rx + 2].reshape(4, C).sum(0) / 4)
+    O, _ = orc.bra_attend(Q, K, V, index, None, heads, S, 0.3)
+    ref = masked_attention_loops(hand_padded(Q, S), Kp, hand_padded(V, S), index, heads, S, 0.3)
+    np.testing.assert_allclose(O, ref[:, :H, :W], rtol=1e-11, atol=1e-12)
+
+
+def test_padded_backward_matches_central_finite_differences():
+    B, H, W, C, heads, S, k = 1, 5, 7, 4, 2, 2, 2
+    g = rng(44)
+    Q, K, V, dO = (g.standard_normal((B, H, W, C)) for _ in range(4))
+    w = 0.3 * g.standard_normal((C, 5, 5))
+    _, _, index, _ = orc.bra_route(Q, K, heads, S, k)
+    grads = orc.bra_backward(Q, K, V, index, w, dO, heads, S, 0.45)
+    assert all(a.shape == Q.shape for a in grads[:3])
+
+    def loss(Q, K, V, w):
+        O, _ = orc.bra_attend(Q, K, V, index, w, heads, S, 0.45)
+        return float((O * dO).sum())
+    eps = 1e-6
+    args = [Q, K, V, w]
+    for a_i, grad in enumerate(grads[:4]):
+        flat = args[a_i].reshape(-1)
+        for p in rng(45 + a_i).choice(flat.size, size=16, replace=False):
+            old = flat[p]
+            flat[p] = old + eps
+            up = loss(*args)
+            flat[p] = old - eps
+            dn = loss(*args)
+            flat[p] = old
+            assert grad.reshape(-1)[p] == pytest.approx((up - dn) / (2 * eps), rel=2e-6, abs=2e-8)
+
+
 # ---------------------------------------------------------------- planted mistakes
 def _sum_for_mean(X, S):
     return orc.region_partition(np.asarray(X, dtype=np.float64), S).sum(axis=2)
@@ -496,7 +579,19 @@ def _dropped_lce_adjoint(real):
     return f
 
 
+def _pad_at_top_left(real):
+    def f(X, S):
+        X = np.asarray(X, dtype=np.float64)
+        Hp, Wp = orc.padded_size(X.shape[1], X.shape[2], S)
+        out = np.zeros((X.shape[0], Hp, Wp, X.shape[3]))
+        out[:, Hp - X.shape[1]:, Wp - X.shape[2]:] = X
+        return out
+    return f
+
+
 PLANTED = [
+    ("pad_map", _pad_at_top_left, ["test_pad_and_crop_place_every_token_by_hand",
+                                   "test_padded_routing_pools_the_zero_tokens_and_matches_the_whole_map_scan"]),
     # (oracle attribute, sabotage, pins of which at least the first must fail)
     ("region_means", lambda real: _sum_for_mean, ["test_affinity_is_mean_of_all_token_pair_products"]),
     ("region_affinity", _transposed_affinity, ["test_affinity_is_mean_of_all_token_pair_products"]),

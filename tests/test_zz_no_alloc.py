@@ -41,8 +41,11 @@ def test_too_large_problem_is_refused_on_the_host(bra):
     assert rc == 11
     assert "no-allocation" in lib.bra_status_string(rc).decode()
     # the usual host checks still come first
-    bad = bra.make_problem(B=1, H=16, W=16, C=64, heads=2, S=3, topk=1)
+    bad = bra.make_problem(B=1, H=16, W=16, C=64, heads=2, S=0, topk=1)
     assert lib.bra_route_static(ctypes.byref(bad), A, A, A, None) == 2
+    # a map S does not divide would need a padded copy of Q and K, i.e. scratch: not through this entry point
+    odd = bra.make_problem(B=1, H=16, W=16, C=64, heads=2, S=3, topk=1)
+    assert lib.bra_route_static(ctypes.byref(odd), A, A, A, None) == 7
     ok = bra.make_problem(B=1, H=16, W=16, C=64, heads=2, S=4, topk=1)
     assert lib.bra_route_static(ctypes.byref(ok), A, None, A, None) == 1
     assert lib.bra_route_static(ctypes.byref(ok), A, A, A + 4, None) == 5
