@@ -15,7 +15,9 @@
  *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte
  *     aligned, dense and contiguous.  The library allocates no device memory
  *     and keeps no state between calls besides kernel attributes and launch
- *     choices remembered per device and problem shape.
+ *     choices remembered per device and problem shape, and one helper stream
+ *     with two events per device and host thread (created by the first
+ *     bra_backward call; its work is forked from and joined back into `stream`).
  *   - Q, K, V, O, dO, dQ, dK, dV: [B, H, W, C], element type p->dtype, channel
  *     c = head * (C / heads) + j (concat order of Eq. 2).
  *   - Regions: S x S non-overlapping blocks of (H/S) x (W/S) tokens, numbered

@@ -434,6 +434,28 @@ bool backward_supported(const Dims& d) {
     return (d.d == 16 || d.d == 32 || d.d == 64) && d.R <= 1000;
 }
 
+// The LCE weight gradient needs only V and dO, the attention gradients need neither of its results: the two
+// run side by side.  A helper stream per device and host thread, forked from and joined back into the
+// caller's stream with events (created on first use; nullptr if that fails, then everything stays in order
+// on the caller's stream).  BRA_NO_SIDE_STREAM keeps the single stream (debugging aid).
+struct SideStream { cudaStream_t s; cudaEvent_t fork, join; };
+static SideStream* side_stream() {
+    static const bool off = getenv("BRA_NO_SIDE_STREAM") != nullptr;
+    if (off) return nullptr;
+    static thread_local SideStream made[64];
+    static thread_local int state[64] = {};            // 0: not tried, 1: ready, 2: failed
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (state[dev] == 0) {
+        SideStream& m = made[dev];
+        const bool ok = cudaStreamCreateWithFlags(&m.s, cudaStreamNonBlocking) == cudaSuccess &&
+                        cudaEventCreateWithFlags(&m.fork, cudaEventDisableTiming) == cudaSuccess &&
+                        cudaEventCreateWithFlags(&m.join, cudaEventDisableTiming) == cudaSuccess;
+        state[dev] = ok ? 1 : 2;
+    }
+    return state[dev] == 1 ? &made[dev] : nullptr;
+}
+
 template <typename T, int D>
 static cudaError_t launch_bwd_t(const Dims& d, int impl, const void* Q, const void* K, const void* V,
                                 const int32_t* index, const float* lce_w, const float* lse,
@@ -448,6 +470,39 @@ static cudaError_t launch_bwd_t(const Dims& d, int impl, const void* Q, const vo
     const T* q = static_cast<const T*>(Q); const T* k = static_cast<const T*>(K);
     const T* v = static_cast<const T*>(V); const T* go = static_cast<const T*>(dO);
     cudaError_t e;
+
+    // ---- LCE weight / bias gradient, beside the attention gradients ----
+    SideStream* ss = (d.lce || d_lce_b) ? side_stream() : nullptr;
+    cudaStream_t dw_st = st;
+    if (ss) {
+        if (cudaEventRecord(ss->fork, st) != cudaSuccess || cudaStreamWaitEvent(ss->s, ss->fork, 0) != cudaSuccess) ss = nullptr;
+        else dw_st = ss->s;
+    }
+    if (d.lce || d_lce_b) {
+        const long long rows = (long long)d.B * d.H;
+        const int rpb = (int)((rows + L.dw_blocks - 1) / L.dw_blocks);
+        const int nblk = (int)((rows + rpb - 1) / rpb);
+        const int cpx = d.C / 2 < DW_CP ? d.C / 2 : DW_CP;
+        const size_t dw_smem = (size_t)(2 * rpb + 4) * d.W * d.C * sizeof(T);
+        if (dw_smem <= 100 * 1024 && ((size_t)d.W * d.C * sizeof(T)) % 16 == 0) {
+            static PerDeviceMax dw_set;
+            if (dw_smem > 48 * 1024 &&
+                (e = dw_set.ensure((int)dw_smem, [&] {
+                     return cudaFuncSetAttribute(bwd_dw_partial_staged_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)dw_smem);
+                 })) != cudaSuccess)
+                return e;
+            bwd_dw_partial_staged_kernel<T><<<nblk, dim3(cpx, DW_TI), dw_smem, dw_st>>>(v, go, part, rpb, d);
+        } else {
+            bwd_dw_partial_kernel<T><<<nblk, dim3(cpx, DW_TI), 0, dw_st>>>(v, go, part, rpb, d);
+        }
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        bwd_dw_final_kernel<<<(d.C * 26 + 31) / 32, dim3(32, DW_SLICES), 0, dw_st>>>(part, nblk, d.lce ? d_lce_w : nullptr, d_lce_b, d);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    if (ss && cudaEventRecord(ss->join, ss->s) != cudaSuccess) return cudaErrorUnknown;
 
     // bf16, head dim 32: tensor-core kernels.  Small maps with enough (image, head) pairs to fill the
     // GPU keep a whole slice resident; the rest stream blocks through shared memory.
@@ -484,30 +539,7 @@ static cudaError_t launch_bwd_t(const Dims& d, int impl, const void* Q, const vo
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
 
-    if (d.lce || d_lce_b) {
-        const long long rows = (long long)d.B * d.H;
-        const int rpb = (int)((rows + L.dw_blocks - 1) / L.dw_blocks);
-        const int nblk = (int)((rows + rpb - 1) / rpb);
-        const int cpx = d.C / 2 < DW_CP ? d.C / 2 : DW_CP;
-        const size_t dw_smem = (size_t)(2 * rpb + 4) * d.W * d.C * sizeof(T);
-        if (dw_smem <= 100 * 1024 && ((size_t)d.W * d.C * sizeof(T)) % 16 == 0) {
-            static PerDeviceMax dw_set;
-            if (dw_smem > 48 * 1024 &&
-                (e = dw_set.ensure((int)dw_smem, [&] {
-                     return cudaFuncSetAttribute(bwd_dw_partial_staged_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 (int)dw_smem);
-                 })) != cudaSuccess)
-                return e;
-            bwd_dw_partial_staged_kernel<T><<<nblk, dim3(cpx, DW_TI), dw_smem, st>>>(v, go, part, rpb, d);
-        } else {
-            bwd_dw_partial_kernel<T><<<nblk, dim3(cpx, DW_TI), 0, st>>>(v, go, part, rpb, d);
-        }
-        count_launch();
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        bwd_dw_final_kernel<<<(d.C * 26 + 31) / 32, dim3(32, DW_SLICES), 0, st>>>(part, nblk, d.lce ? d_lce_w : nullptr, d_lce_b, d);
-        count_launch();
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    }
+    if (ss && cudaStreamWaitEvent(st, ss->join, 0) != cudaSuccess) return cudaErrorUnknown;
     return cudaSuccess;
 }
 
