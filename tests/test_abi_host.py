@@ -37,11 +37,11 @@ def test_library_exports_every_declared_symbol(lib):
 def test_version_and_status_strings(lib):
     assert lib.bra_version() >= 100
     seen = set()
-    for code in range(0, 11):
+    for code in range(0, 12):                     # BRA_OK .. BRA_ERR_STATIC_LIMIT
         s = lib.bra_status_string(code).decode()
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 11
+    assert len(seen) == 12
     assert lib.bra_status_string(99).decode() == "unknown status"
 
 
@@ -117,6 +117,23 @@ def test_null_alignment_workspace_checks(lib):
     bad = list(args); bad[6] = None                                           # dO
     assert lib.bra_backward(ref, *bad, A, need, None) == 1
     assert lib.bra_device_status(None, None) == 1
+
+
+def test_workspace_init_checks_its_arguments(lib):
+    from paper_2303_08810_b200 import binding
+    p = problem()
+    need = binding.workspace_bytes(p)
+    assert lib.bra_workspace_init(ctypes.byref(p), None, need, None) == 1
+    assert lib.bra_workspace_init(ctypes.byref(p), A + 8, need, None) == 5
+    assert lib.bra_workspace_init(ctypes.byref(p), A, need - 1, None) == 6
+    bad = problem(S=0)
+    assert lib.bra_workspace_init(ctypes.byref(bad), A, need, None) == 2
+
+
+def test_injection_switch_is_validated(lib):
+    p = problem()
+    p.inject = 5
+    assert lib.bra_attend(ctypes.byref(p), A, A, A, A, A, None, A, None, A, 1 << 30, None) == 7
 
 
 def test_unsupported_impl_for_problem(lib):
