@@ -180,15 +180,15 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
             if (warp == 0) ok = mbar_wait(bar_s, n_mma & 1, POLL_LIMIT);
             if (!__syncthreads_and(ok)) { ok = false; break; }
             tc_fence_after_sync();
-            // pass 1: row maximum over the 128 keys of the block
+            // pass 1: row maximum over the 128 keys of the block, 32 columns per round trip to tensor memory
             float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll 1
-            for (int cc = 0; cc < 128; cc += 16) {
-                uint32_t r[16];
-                tmem_ld_32x32b_x16(tg + cc, r);
+            for (int cc = 0; cc < 128; cc += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(tg + cc, r);
                 tmem_ld_wait();
 #pragma unroll
-                for (int q = 0; q < 16; q += 4) {
+                for (int q = 0; q < 32; q += 4) {
                     m0 = fmax3(m0, __uint_as_float(r[q]), __uint_as_float(r[q + 1]));
                     m1 = fmax3(m1, __uint_as_float(r[q + 2]), __uint_as_float(r[q + 3]));
                 }
@@ -202,19 +202,22 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
             const float2 sl2v = make_float2(sl2, sl2), mnegv = make_float2(mneg, mneg);
             float2 sum2 = make_float2(0.f, 0.f);
             if (valid) {
-#pragma unroll 1
-                for (int cc = 0; cc < 128; cc += 16) {
-                    uint32_t r[16], pk[8];
-                    tmem_ld_32x32b_x16(tg + cc, r);
+                // loads from tensor memory are issued one step ahead of their use
+                uint32_t r[2][16];
+                tmem_ld_32x32b_x16(tg, r[0]);
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch) {
                     tmem_ld_wait();
+                    if (ch < 7) tmem_ld_32x32b_x16(tg + 16 * (ch + 1), r[(ch + 1) & 1]);
+                    uint32_t pk[8];
 #pragma unroll
                     for (int q = 0; q < 16; q += 2) {
-                        const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[q]), __uint_as_float(r[q + 1])), sl2v, mnegv);
+                        const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[ch & 1][q]), __uint_as_float(r[ch & 1][q + 1])), sl2v, mnegv);
                         const float2 pe = make_float2(ex2w(a.x), ex2w(a.y));
                         sum2 = __fadd2_rn(sum2, pe);
                         pk[q >> 1] = packw(pe.x, pe.y);
                     }
-                    tmem_st_32x32b_x8(tg + (cc >> 1), pk);
+                    tmem_st_32x32b_x8(tg + 8 * ch, pk);
                 }
             } else {                                 // a bad routing entry (the whole CTA sees it): P = 0
                 uint32_t pk[8];
