@@ -335,7 +335,15 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
             ok = wait_count(fw.ctrl + 11, dm.B * dm.heads * ((dm.R + 15) >> 4), polls);
         }
     } else {
-        pdl_wait();                         // the routing index comes from the kernel before (a forward call)
+        // Q and the halo are inputs of the call: their copies overlap the tail of the kernel before (routing,
+        // in a forward call); only the routing index, hence K and V, has to wait for it
+        if (tid == 0 && my_tiles > 0) {
+            mbar_expect_tx_only(bar_qk, k1::QK_BYTES / 2);
+            tma_load_4d(sm_base + OFF_Q, &maps.q, bar_qk, t.c0, t.x0, t.y0, t.b);
+            tma_load_4d(sm_base + OFF_Q + 4096, &maps.q, bar_qk, t.c0 + 32, t.x0, t.y0, t.b);
+            issue_halo(t, 0);
+        }
+        pdl_wait();                         // the routing index comes from the kernel before
     }
     int2 ent = make_int2(0, 0);             // routing entries (head A, head B) of the tile in hand
     int2 raw_n = make_int2(0, 0);           // those of the next tile, as loaded (not yet looked at)
@@ -348,9 +356,18 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
     if (run_tiles > 0) {
         ent = checked(load_entries(t.b, t.i, t.hp));
         if (tid == 0) {
-            issue_qk(t, ent, 0);
+            if (FORWARD) {
+                issue_qk(t, ent, 0);
+                issue_halo(t, 0);
+            } else {                            // Q and the halo are on their way already: K completes the phase
+                const int ra = ent.x < 0 ? 0 : ent.x, rb = ent.y < 0 ? 0 : ent.y;
+                const int rya = (ra * inv_s) >> 20, ryb = (rb * inv_s) >> 20;
+                last_qk = 0;
+                mbar_expect_tx(bar_qk, k1::QK_BYTES / 2);
+                tma_load_4d(sm_base + OFF_K, &maps.k, bar_qk, t.c0, (ra - rya * dm.S) * RS, rya * RS, t.b);
+                tma_load_4d(sm_base + OFF_K + 4096, &maps.k, bar_qk, t.c0 + 32, (rb - ryb * dm.S) * RS, ryb * RS, t.b);
+            }
             issue_v(t, ent, 0);
-            issue_halo(t, 0);
             ok = mbar_wait(bar_qk, 0, POLL_LIMIT);
             if (ok) issue_s();
         }
