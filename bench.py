@@ -16,7 +16,8 @@ shape the headline metric is quoted on).  Prints ONE JSON line.
              one launch / its mean duration from CUDA events (a loop of
              bra_attend calls), against the measured HBM copy bandwidth
   per_shape  the other benchmark shapes (configs 3, 4, 5 and the config-5
-             backward), timed in the same process
+             backward) and the Appendix-D ViT-adaptation shape (config 6, head
+             dim 64), timed in the same process
   cpu_baseline  the fp64 CPU oracle timed on a bounded sample (rank 0, N=1):
              one thread, and the same sample split over all host cores
 
@@ -451,7 +452,7 @@ def main():
     per_shape = None
     if not args.no_per_shape and args.config == 2 and rank == 0:
         per_shape = []
-        for number in (3, 4, 5):
+        for number in (3, 4, 5, 6):
             other = Workload(number, rank, dev)
             per_shape.append(shape_report(other, 50, 3, peak, peak_tf, peak_kind, rank))
             del other

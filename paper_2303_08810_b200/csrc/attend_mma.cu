@@ -1,5 +1,5 @@
 // Routed token-to-token attention + LCE with warp-level tensor-core MMAs
-// (Eq. 6, Eq. 7 with Eq. 1): head dim 32, bf16, any region shape and any topk.
+// (Eq. 6, Eq. 7 with Eq. 1): head dim 32 or 64, bf16, any region shape and any topk.
 //
 // tcgen05 MMAs work on 128-row tiles; a BRA query group is one region's n_r tokens of one
 // head, each group with its own routed keys, so for small regions (n_r = 4 or 16) a 128-row
@@ -17,12 +17,16 @@
 //   3. normalised O^att to an fp32 staging tile (over the dead K/V buffers).
 //   4. all threads: LCE from the halo tile (thread = channel pair x run of 2 tokens),
 //      + O^att, bf16 store of O.
+// A head of 64 channels (template parameter PL = 2) is handled as two planes of 32: every tile
+// (Q, K, V, halo, staging) exists once per plane in the layout above, S sums the two planes'
+// products, O and the LCE run per plane.
 #include "mma_common.cuh"
 
 namespace bra {
 
 using namespace ptx;
 
+template <int PL>
 __global__ void __launch_bounds__(wm::MAXW * 32)
 attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __restrict__ Kg,
                   const __nv_bfloat16* __restrict__ Vg, const int32_t* index,
@@ -49,7 +53,7 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
     const size_t tok_bytes = (size_t)dm.C * 2;
     const size_t row_bytes = (size_t)dm.W * tok_bytes;
     const size_t img = (size_t)b * dm.H * row_bytes;
-    const size_t ch_off = (size_t)h * 64;                             // this head's 32 channels
+    const size_t ch_off = (size_t)h * 64 * PL;                        // this head's 32 * PL channels
     const uint8_t* Qb = reinterpret_cast<const uint8_t*>(Qg) + img + ch_off;
     const uint8_t* Kb = reinterpret_cast<const uint8_t*>(Kg) + img + ch_off;
     const uint8_t* Vb = reinterpret_cast<const uint8_t*>(Vg) + img + ch_off;
@@ -69,14 +73,17 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
 
     // ---- loaders ----
     // one row = one token's 64 bytes of this head = 4 chunks of 16 B, chunk index xor (row >> 1) & 3
-    auto load_row = [&](uint32_t dst_row, int row, const uint8_t* src, bool valid) {
+    // (per plane: the next 64 bytes of the token, `plane_bytes` further on in shared memory)
+    auto load_row = [&](uint32_t dst_row, int row, const uint8_t* src, bool valid, uint32_t plane_bytes) {
         const uint32_t sw = (row >> 1) & 3;
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-            cp_async_16(dst_row + ((q ^ sw) << 4), valid ? src + q * 16 : Kb, valid ? 16u : 0u);
+        for (int p = 0; p < PL; ++p)
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                cp_async_16(dst_row + p * plane_bytes + ((q ^ sw) << 4), valid ? src + p * 64 + q * 16 : Kb, valid ? 16u : 0u);
     };
     auto load_kv_block = [&](int blk, int stage) {
-        const uint32_t kdst = sbase + gm.off_kv + stage * 8192, vdst = kdst + 4096;
+        const uint32_t kdst = sbase + gm.off_kv + stage * (8192 * PL), vdst = kdst + 4096 * PL;
         for (int key = tid; key < KB; key += nthreads) {
             const int kk = blk * KB + key;
             bool valid = kk < total_keys;
@@ -92,8 +99,8 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
                 }
             }
             s_flag[stage * KB + key] = valid ? 1 : 0;
-            load_row(kdst + key * 64, key, Kb + off, valid);
-            load_row(vdst + key * 64, key, Vb + off, valid);
+            load_row(kdst + key * 64, key, Kb + off, valid, 4096);
+            load_row(vdst + key * 64, key, Vb + off, valid, 4096);
         }
     };
     // Q rows of the chunk (rows beyond the region are zero)
@@ -101,7 +108,8 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
         const int t = t0 + row;
         const bool valid = t < dm.n_r;
         const int ty = fdiv(valid ? t : 0, dm.ws, gm.mul_ws), tx = (valid ? t : 0) - ty * dm.ws;
-        load_row(sbase + gm.off_q + row * 64, row, Qb + (size_t)(y0 + ty) * row_bytes + (size_t)(x0 + tx) * tok_bytes, valid);
+        load_row(sbase + gm.off_q + row * 64, row, Qb + (size_t)(y0 + ty) * row_bytes + (size_t)(x0 + tx) * tok_bytes, valid,
+                 gm.nw * 16 * 64);
     }
     // V halo of the chunk's token rows: [rows + 4][ws + 4] tokens x 64 B, zeros outside the map
     const int cy0 = fdiv(t0, dm.ws, gm.mul_ws);                       // first / last region row of the chunk
@@ -116,7 +124,10 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
             const uint8_t* src = Vb + (size_t)(valid ? y : 0) * row_bytes + (size_t)(valid ? x : 0) * tok_bytes;
             const uint32_t dst = sbase + gm.off_halo + cell * 64;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) cp_async_16(dst + q * 16, valid ? src + q * 16 : Vb, valid ? 16u : 0u);
+            for (int p = 0; p < PL; ++p)
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    cp_async_16(dst + p * (gm.halo_rows * gm.halo_w * 64) + q * 16, valid ? src + p * 64 + q * 16 : Vb, valid ? 16u : 0u);
         }
     }
     load_kv_block(0, 0);
@@ -126,12 +137,14 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
     const int g = lane >> 2, tq = lane & 3;                           // fragment row / column pair
     const float sl2 = dm.scale * 1.4426950408889634f;
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    float o[4][4];
+    float o[PL][4][4];
 #pragma unroll
-    for (int n = 0; n < 4; ++n)
+    for (int p = 0; p < PL; ++p)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) o[n][e] = 0.f;
-    uint32_t qa[2][4];
+        for (int n = 0; n < 4; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) o[p][n][e] = 0.f;
+    uint32_t qa[PL][2][4];
     const bool lower_only = (t1 - t0) - warp * 16 <= 8;               // rows g + 8 of this warp are padding
 
     for (int blk = 0; blk < gm.nblocks; ++blk) {
@@ -148,23 +161,28 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
             // A fragments of Q: ldmatrix x4 per k-step: (rows 0-7, ch lo), (rows 8-15, ch lo), (rows 0-7, ch hi), (rows 8-15, ch hi)
             const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-            for (int s = 0; s < 2; ++s) {
-                const int q = 2 * s + (lane >> 4);
-                ldmatrix_x4(sbase + gm.off_q + row * 64 + ((q ^ ((row >> 1) & 3)) << 4), qa[s]);
-            }
+            for (int p = 0; p < PL; ++p)
+#pragma unroll
+                for (int s = 0; s < 2; ++s) {
+                    const int q = 2 * s + (lane >> 4);
+                    ldmatrix_x4(sbase + gm.off_q + p * (gm.nw * 16 * 64) + row * 64 + ((q ^ ((row >> 1) & 3)) << 4), qa[p][s]);
+                }
         }
-        const uint32_t kbase = sbase + gm.off_kv + stage * 8192, vbase = kbase + 4096;
+        const uint32_t kbase = sbase + gm.off_kv + stage * (8192 * PL), vbase = kbase + 4096 * PL;
         // S = Q K^T: 8 key tiles of 8
         float c[8][4];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
-            uint32_t kb[4];
             const int key = 8 * j + (lane & 7);
             const int q = lane >> 3;                                  // channel chunk of this lane's matrix
-            ldmatrix_x4(kbase + key * 64 + ((q ^ ((key >> 1) & 3)) << 4), kb);
-            mma_bf16(c[j], qa[0], kb[0], kb[1]);
-            mma_bf16(c[j], qa[1], kb[2], kb[3]);
+#pragma unroll
+            for (int p = 0; p < PL; ++p) {
+                uint32_t kb[4];
+                ldmatrix_x4(kbase + p * 4096 + key * 64 + ((q ^ ((key >> 1) & 3)) << 4), kb);
+                mma_bf16(c[j], qa[p][0], kb[0], kb[1]);
+                mma_bf16(c[j], qa[p][1], kb[2], kb[3]);
+            }
         }
         // keys that do not count (padding of the last block, out-of-range entries): -inf
         const uint8_t* fl = s_flag + stage * KB;
@@ -195,7 +213,9 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
             l_run[r] *= corr[r];
         }
 #pragma unroll
-        for (int n = 0; n < 4; ++n) { o[n][0] *= corr[0]; o[n][1] *= corr[0]; o[n][2] *= corr[1]; o[n][3] *= corr[1]; }
+        for (int p = 0; p < PL; ++p)
+#pragma unroll
+            for (int n = 0; n < 4; ++n) { o[p][n][0] *= corr[0]; o[p][n][1] *= corr[0]; o[p][n][2] *= corr[1]; o[p][n][3] *= corr[1]; }
         uint32_t pa[4][4];                                            // P as A fragments: 4 k-steps of 16 keys
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -216,13 +236,15 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
         for (int s = 0; s < 4; ++s) {
             const int key = 16 * s + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-            for (int np = 0; np < 2; ++np) {
-                uint32_t vb[4];
-                const int q = 2 * np + (lane >> 4);
-                ldmatrix_x4_trans(vbase + key * 64 + ((q ^ ((key >> 1) & 3)) << 4), vb);
-                mma_bf16(o[2 * np], pa[s], vb[0], vb[1]);
-                mma_bf16(o[2 * np + 1], pa[s], vb[2], vb[3]);
-            }
+            for (int p = 0; p < PL; ++p)
+#pragma unroll
+                for (int np = 0; np < 2; ++np) {
+                    uint32_t vb[4];
+                    const int q = 2 * np + (lane >> 4);
+                    ldmatrix_x4_trans(vbase + p * 4096 + key * 64 + ((q ^ ((key >> 1) & 3)) << 4), vb);
+                    mma_bf16(o[p][2 * np], pa[s], vb[0], vb[1]);
+                    mma_bf16(o[p][2 * np + 1], pa[s], vb[2], vb[3]);
+                }
         }
         __syncthreads();                                              // this stage may be overwritten
     }
@@ -241,9 +263,11 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
         if (t < dm.n_r) {
             const float inv = l_run[r] > 0.f ? 1.f / l_run[r] : 0.f;
 #pragma unroll
-            for (int n = 0; n < 4; ++n)
-                *reinterpret_cast<float2*>(stage_o + row * 32 + 8 * n + 2 * tq) =
-                    make_float2(o[n][2 * r] * inv, o[n][2 * r + 1] * inv);
+            for (int p = 0; p < PL; ++p)
+#pragma unroll
+                for (int n = 0; n < 4; ++n)
+                    *reinterpret_cast<float2*>(stage_o + p * (gm.nw * 16 * 32) + row * 32 + 8 * n + 2 * tq) =
+                        make_float2(o[p][n][2 * r] * inv, o[p][n][2 * r + 1] * inv);
             if (lse && tq == 0) {
                 const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
                 lse[((size_t)b * dm.heads + h) * dm.N + (size_t)(y0 + ty) * dm.W + x0 + tx] =
@@ -258,45 +282,50 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
         const int cp = tid & 15;                                      // channels 2cp, 2cp + 1 of this head
         const int run = (dm.ws & 1) ? 1 : 2;
         const int nruns = (t1 - t0) / run;                            // chunk boundaries are multiples of 16 or n_r
-        float2 wv[25];
-        float2 bias2 = make_float2(0.f, 0.f);
-        if (dm.lce) {
-            const float* wp = lce_w + (size_t)(h * 32 + 2 * cp) * 25;
-#pragma unroll
-            for (int q = 0; q < 25; ++q) wv[q] = make_float2(__ldg(wp + q), __ldg(wp + 25 + q));
-            if (lce_b) bias2 = make_float2(__ldg(lce_b + h * 32 + 2 * cp), __ldg(lce_b + h * 32 + 2 * cp + 1));
-        }
-        const uint32_t halo = sbase + gm.off_halo + cp * 4;
-        uint32_t* out = reinterpret_cast<uint32_t*>(O) + (img + ch_off) / 4 + cp;
-        for (int u = tid >> 4; u < nruns; u += nthreads >> 4) {
-            const int t = t0 + u * run;
-            const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
-            float2 acc[2] = {bias2, bias2};
+#pragma unroll 1
+        for (int p = 0; p < PL; ++p) {                                // one 32-channel plane of the head at a time
+            const int hc = (h * PL + p) * 32;                         // first channel of the plane
+            float2 wv[25];
+            float2 bias2 = make_float2(0.f, 0.f);
             if (dm.lce) {
+                const float* wp = lce_w + (size_t)(hc + 2 * cp) * 25;
 #pragma unroll
-                for (int ti = 0; ti < 5; ++ti) {
-                    const uint32_t hrow = halo + ((ty - cy0 + ti) * gm.halo_w + tx) * 64;
-                    float2 v[6];
+                for (int q = 0; q < 25; ++q) wv[q] = make_float2(__ldg(wp + q), __ldg(wp + 25 + q));
+                if (lce_b) bias2 = make_float2(__ldg(lce_b + hc + 2 * cp), __ldg(lce_b + hc + 2 * cp + 1));
+            }
+            const uint32_t halo = sbase + gm.off_halo + p * (gm.halo_rows * gm.halo_w * 64) + cp * 4;
+            const float* stage_p = stage_o + p * (gm.nw * 16 * 32);
+            uint32_t* out = reinterpret_cast<uint32_t*>(O) + (img + ch_off) / 4 + p * 16 + cp;
+            for (int u = tid >> 4; u < nruns; u += nthreads >> 4) {
+                const int t = t0 + u * run;
+                const int ty = fdiv(t, dm.ws, gm.mul_ws), tx = t - ty * dm.ws;
+                float2 acc[2] = {bias2, bias2};
+                if (dm.lce) {
 #pragma unroll
-                    for (int xx = 0; xx < 6; ++xx) {
-                        if (xx < run + 4) {
-                            const uint32_t w = lds_u32(hrow + xx * 64);
-                            v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+                    for (int ti = 0; ti < 5; ++ti) {
+                        const uint32_t hrow = halo + ((ty - cy0 + ti) * gm.halo_w + tx) * 64;
+                        float2 v[6];
+#pragma unroll
+                        for (int xx = 0; xx < 6; ++xx) {
+                            if (xx < run + 4) {
+                                const uint32_t w = lds_u32(hrow + xx * 64);
+                                v[xx] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+                            }
+                        }
+#pragma unroll
+                        for (int tj = 0; tj < 5; ++tj) {
+                            acc[0] = __ffma2_rn(wv[ti * 5 + tj], v[tj], acc[0]);
+                            if (run == 2) acc[1] = __ffma2_rn(wv[ti * 5 + tj], v[tj + 1], acc[1]);
                         }
                     }
-#pragma unroll
-                    for (int tj = 0; tj < 5; ++tj) {
-                        acc[0] = __ffma2_rn(wv[ti * 5 + tj], v[tj], acc[0]);
-                        if (run == 2) acc[1] = __ffma2_rn(wv[ti * 5 + tj], v[tj + 1], acc[1]);
-                    }
                 }
-            }
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                if (e < run) {
-                    const float2 att = *reinterpret_cast<const float2*>(stage_o + (t - t0 + e) * 32 + 2 * cp);
-                    const float2 r2 = __fadd2_rn(att, acc[e]);
-                    out[((size_t)(y0 + ty) * dm.W + x0 + tx + e) * (dm.C / 2)] = pack2_bf16(r2.x, r2.y);
+                for (int e = 0; e < 2; ++e) {
+                    if (e < run) {
+                        const float2 att = *reinterpret_cast<const float2*>(stage_p + (t - t0 + e) * 32 + 2 * cp);
+                        const float2 r2 = __fadd2_rn(att, acc[e]);
+                        out[((size_t)(y0 + ty) * dm.W + x0 + tx + e) * (dm.C / 2)] = pack2_bf16(r2.x, r2.y);
+                    }
                 }
             }
         }
@@ -305,8 +334,8 @@ attend_mma_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
 
 // ------------------------------------------------------------------ host side
 bool attend_mma_supported(const Dims& d, int dtype) {
-    if (dtype != BRA_BF16 || d.d != 32 || d.topk > wm::KCAP) return false;
-    const MmaGeom g = mma_geom(d);
+    if (dtype != BRA_BF16 || (d.d != 32 && d.d != 64) || d.topk > wm::KCAP) return false;
+    const MmaGeom g = mma_geom(d, d.d / 32);
     // the staging tile sits over the K/V buffers; chunk boundaries must not split a token run of the LCE
     if (g.nw * 2048 > g.stages * 8192) return false;
     if (g.chunks > 1 && ((g.nw * 16) % d.ws) != 0) return false;
@@ -317,16 +346,18 @@ bool attend_mma_supported(const Dims& d, int dtype) {
 cudaError_t launch_attend_mma(const Dims& d, const void* Q, const void* K, const void* V,
                               const int32_t* index, const float* lce_w, const float* lce_b,
                               void* O, float* lse, int32_t* status, cudaStream_t st, bool after_own_kernel) {
-    const MmaGeom g = mma_geom(d);
-    static PerDeviceMax smem_set;
+    const int planes = d.d / 32;
+    const MmaGeom g = mma_geom(d, planes);
+    auto kernel = planes == 2 ? attend_mma_kernel<2> : attend_mma_kernel<1>;
+    static PerDeviceMax smem_set[2];
     cudaError_t e = cudaSuccess;
     if (g.smem_bytes > 48 * 1024)
-        e = smem_set.ensure(g.smem_bytes, [&] {
-            return cudaFuncSetAttribute(attend_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
+        e = smem_set[planes - 1].ensure(g.smem_bytes, [&] {
+            return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem_bytes);
         });
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)((long long)d.B * d.R * d.heads * g.chunks);
-    e = launch_kernel(attend_mma_kernel, dim3(grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st,
+    e = launch_kernel(kernel, dim3(grid), dim3(g.nw * 32), (size_t)g.smem_bytes, st,
                                   after_own_kernel,
                                   static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
                                   static_cast<const __nv_bfloat16*>(V), index, lce_w, lce_b,

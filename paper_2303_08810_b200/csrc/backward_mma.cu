@@ -467,7 +467,7 @@ static BwdGeom bwd_geom(const Dims& d, bool key_centric) {
 }
 
 bool backward_mma_supported(const Dims& d, int dtype) {
-    if (!attend_mma_supported(d, dtype)) return false;
+    if (d.d != 32 || !attend_mma_supported(d, dtype)) return false;      // the gradient kernels are built for head dim 32
     const BwdGeom a = bwd_geom(d, false), b = bwd_geom(d, true);
     return a.smem_bytes <= 200 * 1024 && b.smem_bytes <= 200 * 1024 && b.g.nw * 2048 <= b.g.stages * 8192;
 }

@@ -22,6 +22,7 @@ struct MmaGeom {
     int halo_rows;     // rows of the halo tile (largest chunk) incl. the 4 border rows
     uint32_t mul_nr, mul_ws, mul_s;   // ceil(2^32 / d) for d = n_r, ws, S
     int off_q, off_kv, off_flag, off_idx, off_halo, smem_bytes;
+    int planes;        // 32-channel planes of a head (head dim / 32); every tile below exists once per plane
 };
 
 __device__ __forceinline__ uint32_t fdiv(uint32_t n, uint32_t d, uint32_t mul) {
@@ -64,8 +65,9 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
 // ------------------------------------------------------------------ host side
 inline uint32_t recip32(int d) { return d <= 1 ? 0u : (uint32_t)(((1ull << 32) + (uint64_t)d - 1) / (uint64_t)d); }
 
-inline MmaGeom mma_geom(const Dims& d) {
+inline MmaGeom mma_geom(const Dims& d, int planes = 1) {
     MmaGeom g;
+    g.planes = planes;
     const int rb = (d.n_r + 15) / 16;
     g.nw = rb < wm::MAXW ? rb : wm::MAXW;
     g.chunks = (d.n_r + g.nw * 16 - 1) / (g.nw * 16);
@@ -76,11 +78,11 @@ inline MmaGeom mma_geom(const Dims& d) {
     g.halo_rows = (chunk_rows < d.hs ? chunk_rows : d.hs) + 4;
     g.mul_nr = recip32(d.n_r); g.mul_ws = recip32(d.ws); g.mul_s = recip32(d.S);
     int off = 0;
-    g.off_q = off;    off += g.nw * 16 * 64;
-    g.off_kv = off;   off += g.stages * 8192;                         // also the fp32 staging tile: nw * 2 KB
+    g.off_q = off;    off += planes * g.nw * 16 * 64;
+    g.off_kv = off;   off += planes * g.stages * 8192;                // also the fp32 staging tile: nw * 2 KB per plane
     g.off_flag = off; off += g.stages * wm::KB;
     g.off_idx = off;  off += ((d.topk * 4 + 15) / 16) * 16;
-    g.off_halo = off; off += d.lce ? g.halo_rows * g.halo_w * 64 : 0;
+    g.off_halo = off; off += d.lce ? planes * g.halo_rows * g.halo_w * 64 : 0;
     g.smem_bytes = off;
     return g;
 }

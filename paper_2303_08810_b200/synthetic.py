@@ -64,6 +64,9 @@ CONFIGS = {
     3: BraConfig("biformer-t-stage3", 64, 14, 14, 256, 8, 7, 16, "bf16"),
     4: BraConfig("dense-pred-512", 2, 128, 128, 64, 2, 8, 4, "bf16"),
     5: BraConfig("biformer-t-stage2-train", 64, 28, 28, 128, 4, 7, 4, "bf16", backward=True),
+    # not one of the benchmark's five: the plain-ViT adaptation of Appendix D (DeiT-B width: 12 heads of 64
+    # channels, 32 x 32 map, S = 8, k = 12: 192 keys per query); the batch size is ours
+    6: BraConfig("vit-adaptation", 16, 32, 32, 768, 12, 8, 12, "bf16"),
 }
 
 

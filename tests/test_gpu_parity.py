@@ -267,6 +267,11 @@ MMA_CASES = TC_CASES + [
     BraConfig("mma-7x7-regions-k3", 1, 56, 56, 64, 2, 8, 3, "bf16"),
     BraConfig("mma-one-token-regions", 1, 4, 4, 32, 1, 4, 5, "bf16"),
     BraConfig("mma-wide-regions-3-chunks", 1, 18, 64, 32, 1, 1, 1, "bf16"),
+    # head dim 64: two 32-channel planes per head
+    BraConfig("mma-d64-vit-adaptation", 1, 32, 32, 768, 12, 8, 12, "bf16"),
+    BraConfig("mma-d64-8x8-regions-k2", 2, 16, 16, 128, 2, 2, 2, "bf16"),
+    BraConfig("mma-d64-3x5-regions", 1, 12, 20, 192, 3, 4, 3, "bf16"),
+    BraConfig("mma-d64-last-block-partial", 1, 14, 14, 64, 1, 7, 49, "bf16"),
 ]
 
 
@@ -288,7 +293,7 @@ def test_attend_mma_options(bra):
 
 
 # head dim 32, bf16, maps small enough that one (image, head) of K and V fits in shared memory
-IMG_CASES = [c for c in MMA_CASES if c.H * c.W <= 1500] + [
+IMG_CASES = [c for c in MMA_CASES if c.H * c.W <= 1500 and c.C // c.heads == 32] + [
     BraConfig("img-tail-tile-n_r=24", 2, 12, 16, 64, 2, 2, 3, "bf16"),
     BraConfig("img-5x5-regions-odd", 1, 15, 15, 32, 1, 3, 4, "bf16"),
     BraConfig("img-k-many-blocks", 1, 16, 16, 64, 2, 4, 16, "bf16"),
