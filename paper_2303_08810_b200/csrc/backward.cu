@@ -435,27 +435,7 @@ bool backward_supported(const Dims& d) {
 }
 
 // The LCE weight gradient needs only V and dO, the attention gradients need neither of its results: the two
-// run side by side.  A helper stream per device and host thread, forked from and joined back into the
-// caller's stream with events (created on first use; nullptr if that fails, then everything stays in order
-// on the caller's stream).  BRA_NO_SIDE_STREAM keeps the single stream (debugging aid).
-struct SideStream { cudaStream_t s; cudaEvent_t fork, join; };
-static SideStream* side_stream() {
-    static const bool off = getenv("BRA_NO_SIDE_STREAM") != nullptr;
-    if (off) return nullptr;
-    static thread_local SideStream made[64];
-    static thread_local int state[64] = {};            // 0: not tried, 1: ready, 2: failed
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (state[dev] == 0) {
-        SideStream& m = made[dev];
-        const bool ok = cudaStreamCreateWithFlags(&m.s, cudaStreamNonBlocking) == cudaSuccess &&
-                        cudaEventCreateWithFlags(&m.fork, cudaEventDisableTiming) == cudaSuccess &&
-                        cudaEventCreateWithFlags(&m.join, cudaEventDisableTiming) == cudaSuccess;
-        state[dev] = ok ? 1 : 2;
-    }
-    return state[dev] == 1 ? &made[dev] : nullptr;
-}
-
+// run side by side (helper stream of bra_internal.h; everything stays on the caller's stream if there is none).
 template <typename T, int D>
 static cudaError_t launch_bwd_t(const Dims& d, int impl, const void* Q, const void* K, const void* V,
                                 const int32_t* index, const float* lce_w, const float* lse,

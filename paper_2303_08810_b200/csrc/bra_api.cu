@@ -83,6 +83,23 @@ static bra_status check_ws(const Dims& d, const void* ws, size_t ws_bytes, WsLay
     return BRA_OK;
 }
 
+SideStream* side_stream() {
+    static const bool off = getenv("BRA_NO_SIDE_STREAM") != nullptr;
+    if (off) return nullptr;
+    static thread_local SideStream made[64];
+    static thread_local int state[64] = {};            // 0: not tried, 1: ready, 2: failed
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (state[dev] == 0) {
+        SideStream& m = made[dev];
+        const bool ok = cudaStreamCreateWithFlags(&m.s, cudaStreamNonBlocking) == cudaSuccess &&
+                        cudaEventCreateWithFlags(&m.fork, cudaEventDisableTiming) == cudaSuccess &&
+                        cudaEventCreateWithFlags(&m.join, cudaEventDisableTiming) == cudaSuccess;
+        state[dev] = ok ? 1 : 2;
+    }
+    return state[dev] == 1 ? &made[dev] : nullptr;
+}
+
 static bool padded(const Dims& d) { return d.H != d.H0 || d.W != d.W0; }
 
 // The zero-padded copy of a caller's map in slot `slot` of the scratch buffer (or the map itself if S divides it).

@@ -137,6 +137,12 @@ struct PerDeviceOnce {
     cudaError_t run(F&& set) { return m.ensure(1, set); }
 };
 
+// A helper stream per device and host thread, forked from and joined back into the caller's stream with
+// events (created on first use; nullptr if that fails or BRA_NO_SIDE_STREAM is set: then the work stays in
+// order on the caller's stream).
+struct SideStream { cudaStream_t s; cudaEvent_t fork, join; };
+SideStream* side_stream();
+
 bool backward_supported(const Dims& d);
 // impl: the bra_impl the caller asked for
 cudaError_t launch_backward(const Dims& d, int dtype, int impl, const void* Q, const void* K, const void* V,
