@@ -86,13 +86,13 @@ typedef enum bra_impl {
 
 /*
  * Failure injection for tests of the error path (no GPU fault, trap or hang is involved).
- * BRA_INJECT_HOLD_ROUTE_FLAGS: in the one-launch forward (bra_forward with BRA_IMPL_TC_FUSED) one pooled
+ * BRA_INJECT_LOSE_POOLED_UNIT: in the one-launch forward (bra_forward with BRA_IMPL_TC_FUSED) one pooled
  * unit is never counted as done, so every CTA's bounded wait for the end of the pooling phase runs out
  * after a few thousand polls, before any tensor-core work or tile copy has been issued;
  * the kernel returns normally, O is not written and bra_device_status() reports BRA_ERR_TIMEOUT.
  * Ignored by every other path.
  */
-typedef enum bra_inject { BRA_INJECT_NONE = 0, BRA_INJECT_HOLD_ROUTE_FLAGS = 1 } bra_inject;
+typedef enum bra_inject { BRA_INJECT_NONE = 0, BRA_INJECT_LOSE_POOLED_UNIT = 1 } bra_inject;
 
 /* Problem statement in the notation of Algorithm 1 (H, W, C, S, k) plus batch and heads. */
 typedef struct bra_problem {

@@ -49,7 +49,7 @@ static bra_status make_dims(const bra_problem* p, Dims* out) {
     if (p->dtype != BRA_F32 && p->dtype != BRA_BF16) return BRA_ERR_DTYPE;
     if (p->lce_ksize != 0 && p->lce_ksize != 5) return BRA_ERR_UNSUPPORTED;
     if (p->impl < BRA_IMPL_AUTO || p->impl > BRA_IMPL_TC_FUSED) return BRA_ERR_UNSUPPORTED;
-    if (p->inject != BRA_INJECT_NONE && p->inject != BRA_INJECT_HOLD_ROUTE_FLAGS) return BRA_ERR_UNSUPPORTED;
+    if (p->inject != BRA_INJECT_NONE && p->inject != BRA_INJECT_LOSE_POOLED_UNIT) return BRA_ERR_UNSUPPORTED;
     Dims d;
     d.B = p->B; d.H = Hp; d.W = Wp; d.C = p->C; d.heads = p->heads; d.S = p->S; d.topk = p->topk;
     d.H0 = p->H; d.W0 = p->W;
