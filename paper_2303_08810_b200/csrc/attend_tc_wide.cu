@@ -39,7 +39,8 @@ constexpr int OFF_KV = 8192;                             // 2 x { K [128 keys][6
 constexpr int OFF_HALO = OFF_KV + 2 * 16384;             // [12][20][32 ch] bf16, linear
 constexpr int OFF_BAR = OFF_HALO + HALO_BYTES;
 constexpr int ALIGN = 512;                               // the 64-byte swizzle repeats every 512 bytes
-constexpr int SMEM_BYTES = OFF_BAR + 64 + ALIGN;         // + slack for the manual alignment
+constexpr int OFF_ENT = OFF_BAR + 64;                    // the tile's routing entries (KCAP ints)
+constexpr int SMEM_BYTES = OFF_ENT + KCAP * 4 + ALIGN;   // + slack for the manual alignment
 constexpr uint32_t POLL_LIMIT = 4000000u;
 }  // namespace tw
 
@@ -65,6 +66,9 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
     uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem + OFF_BAR);       // S landed in TMEM
     uint64_t* bar_o = bar_s + 1;                                         // O landed in TMEM
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_s + 2);
+    uint64_t* bar_sh = bar_s + 3;                                        // high half of S landed
+    uint32_t* arrivals = reinterpret_cast<uint32_t*>(bar_s + 4);         // threads that have read O out of tensor memory (running count)
+    volatile int32_t* ent = reinterpret_cast<volatile int32_t*>(smem + OFF_ENT);
     const uint32_t sm_base = smem_u32(smem);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -75,6 +79,8 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
     if (tid == 0) {
         mbar_init(bar_s, 1);
         mbar_init(bar_o, 1);
+        mbar_init(bar_sh, 1);
+        *arrivals = 0;
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(tmem_slot, TMEM_COLS);
@@ -101,11 +107,12 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
     const int cp = lane & 15;
     const int xl0 = 2 * (warp * 2 + (lane >> 4));
 
-    constexpr uint32_t IDESC_S = umma_idesc_bf16(128, 128, false, false);
+    constexpr uint32_t IDESC_SH = umma_idesc_bf16(128, 64, false, false);
     constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 32, false, true);
 
     bool ok = true;
-    uint32_t n_mma = 0;                              // MMA groups waited for so far on each barrier
+    uint32_t n_s = 0, n_o = 0;                       // MMA groups waited for so far on each barrier
+    uint32_t n_arr = 0;                              // rounds of `arrivals` so far
 
     for (int T = blockIdx.x; T < num_tiles && ok; T += gridDim.x) {
         int rem = T;
@@ -123,8 +130,11 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
 
         // key block u = (routed slot m, row block of that region); entry -1: out of range, its P is zero
         // (u = m * RB + kb: the launcher keeps R <= 4096, so r / S is a multiply and a shift)
+        // the tile's routing entries go to shared memory once (coherent loads: the index may come from the kernel
+        // this one overlaps); the first one is also read directly, its copies start before the first barrier
+        if (tid < dm.topk) ent[tid] = __ldcg(irow + tid);
         auto load_unit = [&](int m, int kb, int buf) -> bool {
-            int r = __ldcg(irow + m);        // coherent load: the index may come from the kernel this one overlaps
+            int r = m == 0 ? __ldcg(irow) : ent[m];
             const bool valid = r >= 0 && r < dm.R;
             if (!valid) { record_error(status, BRA_ERR_INDEX, r); r = 0; }
             const int qy = (r * inv_s) >> 20, qx = r - qy * dm.S;
@@ -152,35 +162,32 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
         int m_next = 0, kb_next = 0;             // (routed slot, row block) of the key block being loaded
         cp_async_commit();
 
-        float m_run = -INFINITY, l_run = 0.f;
+        // Softmax over the routed key blocks without a rescaling step per block: the first valid block
+        // fixes the reference maximum m_run (its own row maximum); later blocks use it as it stands, so
+        // their probabilities exp2(s - m_run) may exceed 1.  That is exact as long as nothing overflows
+        // (numerator and denominator carry the same factor); a block whose row sum comes out above 2^40
+        // anywhere in the CTA is done again the slow way: S recomputed, row maximum, m_run raised, the
+        // sums so far rescaled.  With the maximum settled in the first block that path is rare.
+        float m_run = 0.f, l_run = 0.f;
+        bool have_m = false;                         // CTA-uniform: a routing entry is valid or not for the whole tile
         float o_acc[32];
 #pragma unroll
         for (int q = 0; q < 32; ++q) o_acc[q] = 0.f;
 
-        for (int u = 0; u < units; ++u) {
-            const int buf = u & 1;
-            const bool valid = valid_next;
-            cp_async_wait<0>();
-            fence_proxy_async_smem();
-            __syncthreads();                         // block u landed; O of block u - 1 has been read by all
-            if (tid == 0) {
-                tc_fence_after_sync();
-                const uint32_t qa = sm_base + OFF_Q, ka = sm_base + OFF_KV + buf * 16384;
+        // S of a key block is made in two halves of 64 keys, columns [0,64) and [64,128) of tensor memory,
+        // each with its own barrier: the low half of the NEXT block is issued right behind O = P V of this one
+        // (the tensor core takes them in order, and P V is the last reader of those columns), the high half as
+        // soon as every thread has read O out of columns [64,96).  So the threads never wait for an S.
+        auto issue_s_half = [&](int buf, int half) {
+            const uint32_t qa = sm_base + OFF_Q, ka = sm_base + OFF_KV + buf * 16384 + half * 4096;
 #pragma unroll
-                for (int ks = 0; ks < 2; ++ks)       // d = 32 = 2 k-steps of 16
-                    umma_ss(tmem, umma_smem_desc(qa + ks * 32, 16, 512, 4),
-                            umma_smem_desc(ka + ks * 32, 16, 512, 4), IDESC_S, ks);
-                umma_commit(bar_s);
-            }
-            if (u + 1 < units) {                     // next block into the other buffer (its MMAs are done)
-                if (++kb_next == RB) { kb_next = 0; ++m_next; }
-                valid_next = load_unit(m_next, kb_next, buf ^ 1);
-                cp_async_commit();
-            }
-            if (warp == 0) ok = mbar_wait(bar_s, n_mma & 1, POLL_LIMIT);
-            if (!__syncthreads_and(ok)) { ok = false; break; }
-            tc_fence_after_sync();
-            // pass 1: row maximum over the 128 keys of the block, 32 columns per round trip to tensor memory
+            for (int ks = 0; ks < 2; ++ks)           // d = 32 = 2 k-steps of 16
+                umma_ss(tmem + half * 64, umma_smem_desc(qa + ks * 32, 16, 512, 4),
+                        umma_smem_desc(ka + ks * 32, 16, 512, 4), IDESC_SH, ks);
+            umma_commit(half ? bar_sh : bar_s);
+        };
+        // row maximum of S over the 128 keys of the block (raw scores), 32 columns per round trip to tensor memory
+        auto block_max = [&]() -> float {
             float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll 1
             for (int cc = 0; cc < 128; cc += 32) {
@@ -193,63 +200,145 @@ attend_tc_wide_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16*
                     m1 = fmax3(m1, __uint_as_float(r[q + 2]), __uint_as_float(r[q + 3]));
                 }
             }
-            float mx = m_run;
-            if (valid) mx = fmaxf(mx, fmaxf(m0, m1) * sl2);               // sl2 > 0
-            const float corr = (mx == -INFINITY) ? 1.f : ex2w(m_run - mx);
-            const float mneg = (mx == -INFINITY) ? 0.f : -mx;
-            m_run = mx;
-            // pass 2: P = exp2(S * scale * log2 e - max), bf16 pairs over the consumed columns of S; row sum
-            const float2 sl2v = make_float2(sl2, sl2), mnegv = make_float2(mneg, mneg);
+            return fmaxf(m0, m1);
+        };
+        // P = exp2(S * scale * log2 e - m_run) for one half of the block, as bf16 pairs over columns of S
+        // already consumed (half 0: [0,32), half 1: [32,64)); returns the sum over the half's 64 keys.
+        // Loads from tensor memory are issued one step ahead of their use.
+        auto exp_half = [&](int half) -> float {
+            const float2 sl2v = make_float2(sl2, sl2), mnegv = make_float2(-m_run, -m_run);
             float2 sum2 = make_float2(0.f, 0.f);
-            if (valid) {
-                // loads from tensor memory are issued one step ahead of their use
-                uint32_t r[2][16];
-                tmem_ld_32x32b_x16(tg, r[0]);
+            const uint32_t src = tg + 64 * half, dst = tg + 32 * half;
+            uint32_t r[2][16];
+            tmem_ld_32x32b_x16(src, r[0]);
 #pragma unroll
-                for (int ch = 0; ch < 8; ++ch) {
-                    tmem_ld_wait();
-                    if (ch < 7) tmem_ld_32x32b_x16(tg + 16 * (ch + 1), r[(ch + 1) & 1]);
-                    uint32_t pk[8];
+            for (int ch = 0; ch < 4; ++ch) {
+                tmem_ld_wait();
+                if (ch < 3) tmem_ld_32x32b_x16(src + 16 * (ch + 1), r[(ch + 1) & 1]);
+                uint32_t pk[8];
 #pragma unroll
-                    for (int q = 0; q < 16; q += 2) {
-                        const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[ch & 1][q]), __uint_as_float(r[ch & 1][q + 1])), sl2v, mnegv);
-                        const float2 pe = make_float2(ex2w(a.x), ex2w(a.y));
-                        sum2 = __fadd2_rn(sum2, pe);
-                        pk[q >> 1] = packw(pe.x, pe.y);
-                    }
-                    tmem_st_32x32b_x8(tg + 8 * ch, pk);
+                for (int q = 0; q < 16; q += 2) {
+                    const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[ch & 1][q]), __uint_as_float(r[ch & 1][q + 1])), sl2v, mnegv);
+                    const float2 pe = make_float2(ex2w(a.x), ex2w(a.y));
+                    sum2 = __fadd2_rn(sum2, pe);
+                    pk[q >> 1] = packw(pe.x, pe.y);
                 }
+                tmem_st_32x32b_x8(dst + 8 * ch, pk);
+            }
+            return sum2.x + sum2.y;
+        };
+
+        // ---- first key block: wait for it (with Q), issue both halves of its S, start the copy of the second ----
+        cp_async_wait<0>();
+        fence_proxy_async_smem();
+        if (!__syncthreads_and(ok)) { ok = false; break; }
+        if (tid == 0) {
+            tc_fence_after_sync();
+            issue_s_half(0, 0);
+            issue_s_half(0, 1);
+        }
+        bool valid = valid_next;
+        if (units > 1) {
+            if (++kb_next == RB) { kb_next = 0; ++m_next; }
+            valid_next = load_unit(m_next, kb_next, 1);
+            cp_async_commit();
+        }
+
+        for (int u = 0; u < units; ++u) {
+            const int buf = u & 1;
+            const bool more = u + 1 < units;
+            float sum = 0.f;
+            bool big = false;
+            ok = mbar_wait(bar_s, n_s & 1, POLL_LIMIT) && ok;
+            tc_fence_after_sync();
+            if (valid) {
+                if (!have_m) {                       // the first valid block sets the reference maximum
+                    ok = mbar_wait(bar_sh, n_s & 1, POLL_LIMIT) && ok;
+                    tc_fence_after_sync();
+                    m_run = block_max() * sl2;       // sl2 > 0
+                }
+                sum = exp_half(0);
+                ok = mbar_wait(bar_sh, n_s & 1, POLL_LIMIT) && ok;
+                tc_fence_after_sync();
+                sum += exp_half(1);
+                big = !(sum <= 0x1p40f);             // also catches inf and NaN
             } else {                                 // a bad routing entry (the whole CTA sees it): P = 0
+                ok = mbar_wait(bar_sh, n_s & 1, POLL_LIMIT) && ok;
+                tc_fence_after_sync();
                 uint32_t pk[8];
 #pragma unroll
                 for (int q = 0; q < 8; ++q) pk[q] = 0u;
 #pragma unroll 1
                 for (int cc = 0; cc < 64; cc += 8) tmem_st_32x32b_x8(tg + cc, pk);
             }
+            ++n_s;
             tmem_st_wait();
             tc_fence_before_sync();
-            __syncthreads();
+            cp_async_wait<0>();                      // this thread's copies of block u + 1 (issued a block ago)
+            fence_proxy_async_smem();
+            if (__syncthreads_or(big || !ok)) {
+                if (!__syncthreads_and(ok)) { ok = false; break; }   // a wait gave up somewhere: the tile ends here
+                // the slow way: S again (P has overwritten its low half), true row maximum, everything rescaled
+                if (tid == 0) {
+                    tc_fence_after_sync();
+                    issue_s_half(buf, 0);
+                    issue_s_half(buf, 1);
+                }
+                ok = mbar_wait(bar_s, n_s & 1, POLL_LIMIT) && ok;
+                ok = mbar_wait(bar_sh, n_s & 1, POLL_LIMIT) && ok;
+                ++n_s;
+                tc_fence_after_sync();
+                const float m_new = fmaxf(m_run, block_max() * sl2);
+                const float corr = ex2w(m_run - m_new);
+                m_run = m_new;
+                l_run *= corr;
+#pragma unroll
+                for (int q = 0; q < 32; ++q) o_acc[q] *= corr;
+                sum = exp_half(0);
+                sum += exp_half(1);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncthreads();
+            }
+            have_m = have_m || valid;
             if (tid == 0) {
                 tc_fence_after_sync();
                 const uint64_t vd = umma_smem_desc(sm_base + OFF_KV + buf * 16384 + 8192, 16, 512, 4);
-#pragma unroll 1
+#pragma unroll
                 for (int ks = 0; ks < 8; ++ks)       // 128 keys = 8 k-steps of 16 (1024 B of V each)
                     umma_ts(tmem + TM_O, tmem + ks * 8, vd + (uint64_t)(ks * 64), IDESC_O, ks);
                 umma_commit(bar_o);
+                if (more) issue_s_half(buf ^ 1, 0);  // block u + 1 has landed (the barrier above)
             }
-            if (warp == 0) ok = mbar_wait(bar_o, n_mma & 1, POLL_LIMIT);
-            ++n_mma;
-            if (!__syncthreads_and(ok)) { ok = false; break; }
+            ok = mbar_wait(bar_o, n_o & 1, POLL_LIMIT) && ok;
+            ++n_o;
             tc_fence_after_sync();
             uint32_t oraw[32];
             tmem_ld_32x32b_x32(tg + TM_O, oraw);
             tmem_ld_wait();
             tc_fence_before_sync();
-            l_run = fmaf(l_run, corr, sum2.x + sum2.y);
+            l_run += sum;
 #pragma unroll
-            for (int q = 0; q < 32; ++q) o_acc[q] = fmaf(o_acc[q], corr, __uint_as_float(oraw[q]));
+            for (int q = 0; q < 32; ++q) o_acc[q] += __uint_as_float(oraw[q]);
+            if (more) {
+                // columns [64,128) are free once all 128 threads have read O: the last one to say so issues the
+                // high half of the next S (no barrier: the others go straight on to the low half, which is ready)
+                uint32_t before;
+                asm volatile("atom.acq_rel.cta.shared.add.u32 %0, [%1], 1;" : "=r"(before) : "r"(smem_u32(arrivals)) : "memory");
+                if (before == n_arr * THREADS + (THREADS - 1)) {
+                    tc_fence_after_sync();
+                    issue_s_half(buf ^ 1, 1);
+                }
+                ++n_arr;
+                valid = valid_next;
+                if (u + 2 < units) {                 // K and V of block u are done with: block u + 2 takes their place
+                    if (++kb_next == RB) { kb_next = 0; ++m_next; }
+                    valid_next = load_unit(m_next, kb_next, buf);
+                    cp_async_commit();
+                }
+            }
         }
-        if (!ok) break;
+        if (!__syncthreads_and(ok)) { ok = false; break; }   // every thread waits on the barriers itself: agree before going on
 
         // the head's LCE weights for this thread's channel pair: fetched here, not held through the key
         // loop (50 registers); the loads fly during the staging below

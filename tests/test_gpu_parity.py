@@ -163,13 +163,15 @@ IMPLS = {"simt": 1, "mma": 2, "tc": 3, "img": 4, "auto": 0}
 
 
 def run_attend_case(bra, cfg, impl, seed, shared=False, lce=True, bias=False, scale=0.0,
-                    index=None, clustered=False):
+                    index=None, clustered=False, mutate=None):
     """One bra_attend call of kernel family `impl` against the oracle.  A family that is
     named explicitly must take the shape: BRA_ERR_UNSUPPORTED fails the test (the cases
     where a family rightly refuses a shape are asserted in
     test_kernel_families_refuse_only_what_they_should)."""
     import torch
     x = synthetic.make_inputs(cfg, seed=seed, clustered=clustered)
+    if mutate is not None:
+        mutate(x)
     t = to_dev(x, cfg)
     p = problem_of(bra, cfg, impl=IMPLS[impl], shared_routing=shared, lce=lce, scale=scale)
     ws = bra.workspace(p)
@@ -342,6 +344,21 @@ def test_attend_tc_wide_options(bra):
     run_attend_case(bra, cfg, "tc", seed=6, shared=True)
     idx = np.array([[[[3, 3], [0, 1], [2, 0], [1, 1]]] * 2], dtype=np.int32)
     run_attend_case(bra, cfg, "tc", seed=6, index=idx)
+
+
+@pytest.mark.parametrize("order", [[0, 1, 2, 3], [0, 3, 1, 2], [3, 0, 1, 2], [1, 2, 3, 3]])
+@pytest.mark.parametrize("gain", [8.0, 64.0])
+def test_attend_tc_wide_scores_that_grow_late(bra, order, gain):
+    """The keys of one region are scaled up, so that the row maxima of its key blocks lie far above
+    those of the blocks routed before it (by a few hundred at gain 64): whatever reference
+    maximum the kernel carries from earlier blocks, the result must be the plain softmax."""
+    cfg = BraConfig("wide-late-scores", 1, 32, 32, 64, 2, 2, 4, "bf16")
+
+    def louder_region_3(x):
+        x["K"][:, 16:, 16:, :] *= gain             # region 3 of the 2 x 2 partition
+
+    idx = np.array([[[order] * 4] * 2], dtype=np.int32)
+    run_attend_case(bra, cfg, "tc", seed=31, index=idx, mutate=louder_region_3)
 
 
 OPT_CASES = [BraConfig("opts", 2, 16, 16, 64, 2, 4, 3, "bf16"),
