@@ -259,7 +259,7 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
     int hp_loaded = -1;
 
     constexpr uint32_t IDESC_S = umma_idesc_bf16(128, 128, false, false);
-    constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 32, false, true);
+    constexpr uint32_t IDESC_O = umma_idesc_bf16(128, 64, false, true);
 
     auto coord_of = [&](int b, int i, int hp) -> TileCoord {
         TileCoord t;
@@ -446,13 +446,12 @@ attend_tc_k1_kernel(const __grid_constant__ K1Maps maps, const int32_t* index,
             ok = mbar_wait(bar_v, par, POLL_LIMIT);
             if (ok) {
                 tc_fence_after_sync();
+                // one B operand of N = 64 channels: head A's V tile and, 4096 bytes on (the leading-dimension
+                // stride between the two 32-channel atoms), head B's
+                const uint64_t vd = umma_smem_desc(sm_base + OFF_V, k1::OFF_VB - OFF_V, 512, 4);
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const uint64_t vd = umma_smem_desc(sm_base + (hh ? k1::OFF_VB : OFF_V), 16, 512, 4);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)     // 64 keys = 4 k-steps of 16 (1024 B of a V tile each)
-                        umma_ts(tmem + TM_O + hh * 32, tmem + ks * 8, vd + (uint64_t)(ks * 64), IDESC_O, ks);
-                }
+                for (int ks = 0; ks < 4; ++ks)         // 64 keys = 4 k-steps of 16 (1024 B of a V tile each)
+                    umma_ts(tmem + TM_O, tmem + ks * 8, vd + (uint64_t)(ks * 64), IDESC_O, ks);
                 umma_commit(bar_o);
             }
         }
