@@ -272,6 +272,103 @@ route_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ ind
     }
 }
 
+// Routing of one (image, routing head) by one CTA of 256 threads, for R <= 64 regions and 32 channels per
+// routing head - every BiFormer stage with S = 7 or 8.  Three steps with a barrier between them:
+//   1. K^r of the head into shared memory; thread (row i = tid & 63, quarter q = tid >> 6) takes its row of
+//      Q^r into registers;
+//   2. the thread scores candidates j = q, q + 4, ... of its row (Eq. 4: fp32 FMAs over the channels in
+//      increasing order, the sums of the other routing kernels), two candidates at a time so that two
+//      dependent FMA chains are in flight; a warp reads one K^r row at a time (a broadcast); the
+//      order-preserving score bits go to shared memory, [row][65];
+//   3. one thread per row picks the top k (Eq. 5) in k passes over two levels (the best of each group of eight
+//      candidates in registers, a rescan of the winner's group), higher score first, lower region on ties.
+// A warp issues an instruction every five cycles or so in this kind of code, so what counts is the number of
+// instructions one warp runs through: against one thread per row for the scores as well (a single 32-FMA
+// chain per candidate, 49 candidates) the scores are spread over four times the threads.
+constexpr int ROUTE_S_THREADS = 256, ROUTE_S_LD = 36, ROUTE_S_SC = 65;
+
+__global__ void __launch_bounds__(ROUTE_S_THREADS)
+route_small_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ index, Dims dm) {
+    __shared__ __align__(16) float ks[64 * ROUTE_S_LD];
+    __shared__ uint32_t sc[64 * ROUTE_S_SC];
+    pdl_launch_dependents();
+    pdl_wait();                                  // the means come from the kernel before
+    const int tid = threadIdx.x;
+    const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
+    const int c0 = dm.heads_i == 1 ? 0 : h * dm.d;
+    // ---- 1. K^r slice and this thread's row of Q^r (coherent loads: the pooling kernel may still be draining) ----
+    const float* kb = k_mean + (size_t)b * dm.R * dm.C + c0;
+    for (int e = tid; e < dm.R * 8; e += ROUTE_S_THREADS) {
+        const int r = e >> 3, c4 = e & 7;
+        *reinterpret_cast<float4*>(&ks[r * ROUTE_S_LD + 4 * c4]) = __ldcg(reinterpret_cast<const float4*>(kb + (size_t)r * dm.C) + c4);
+    }
+    const int i = tid & 63, q = tid >> 6;
+    float4 qreg[8];
+    {
+        const float4* qrow = reinterpret_cast<const float4*>(q_mean + ((size_t)b * dm.R + (i < dm.R ? i : 0)) * dm.C + c0);
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) qreg[c4] = __ldcg(qrow + c4);
+    }
+    __syncthreads();
+    // ---- 2. scores of candidates q, q + 4, ..., two at a time ----
+    for (int j0 = q; j0 < 64; j0 += 8) {
+        const int j1 = j0 + 4;
+        const float4* ka = reinterpret_cast<const float4*>(&ks[(j0 < dm.R ? j0 : 0) * ROUTE_S_LD]);
+        const float4* kb4 = reinterpret_cast<const float4*>(&ks[(j1 < dm.R ? j1 : 0) * ROUTE_S_LD]);
+        float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 x = ka[c4], y = kb4[c4];
+            a0 = fmaf(qreg[c4].x, x.x, a0); a1 = fmaf(qreg[c4].x, y.x, a1);
+            a0 = fmaf(qreg[c4].y, x.y, a0); a1 = fmaf(qreg[c4].y, y.y, a1);
+            a0 = fmaf(qreg[c4].z, x.z, a0); a1 = fmaf(qreg[c4].z, y.z, a1);
+            a0 = fmaf(qreg[c4].w, x.w, a0); a1 = fmaf(qreg[c4].w, y.w, a1);
+        }
+        // 0 marks "no candidate": real score bits are never 0
+        sc[i * ROUTE_S_SC + j0] = j0 < dm.R ? ordered_bits(a0) : 0u;
+        sc[i * ROUTE_S_SC + j1] = j1 < dm.R ? ordered_bits(a1) : 0u;
+    }
+    __syncthreads();
+    // ---- 3. selection, one thread per row (the other warps are done) ----
+    if (tid >= dm.R) return;
+    uint32_t* row = sc + tid * ROUTE_S_SC;
+    int32_t* out = index + (((size_t)b * dm.heads_i + h) * dm.R + tid) * dm.topk;
+    // Two levels: the best of each group of eight candidates stays in registers; a rank costs a maximum over
+    // the eight group bests and a rescan of the winner's group only.  Strict comparisons in ascending order:
+    // the first of equal scores wins at both levels.
+    uint32_t gbest[8];
+    int garg[8];
+#pragma unroll
+    for (int gq = 0; gq < 8; ++gq) {
+        gbest[gq] = 0u; garg[gq] = 8 * gq;
+#pragma unroll
+        for (int tq = 0; tq < 8; ++tq) {
+            const uint32_t v = row[8 * gq + tq];
+            if (v > gbest[gq]) { gbest[gq] = v; garg[gq] = 8 * gq + tq; }
+        }
+    }
+    for (int m = 0; m < dm.topk; ++m) {
+        uint32_t best = gbest[0];
+        int arg = garg[0];
+#pragma unroll
+        for (int gq = 1; gq < 8; ++gq)
+            if (gbest[gq] > best) { best = gbest[gq]; arg = garg[gq]; }
+        out[m] = arg;
+        row[arg] = 0u;
+        const int wg = arg >> 3;
+        uint32_t nb = 0u;
+        int na = 8 * wg;
+#pragma unroll
+        for (int tq = 0; tq < 8; ++tq) {
+            const uint32_t v = row[8 * wg + tq];
+            if (v > nb) { nb = v; na = 8 * wg + tq; }
+        }
+#pragma unroll
+        for (int gq = 0; gq < 8; ++gq)
+            if (gq == wg) { gbest[gq] = nb; garg[gq] = na; }
+    }
+}
+
 // Routing with one THREAD per affinity row, for larger k: CTA = (image, routing head, chunk of 64
 // rows).  K^r of the head sits in shared memory (read as broadcasts); the thread forms its R scores
 // (Eq. 4: fp32 FMAs over the channels in increasing order, the same sums as the warp-per-row
@@ -524,6 +621,17 @@ static cudaError_t launch_route_rows(const Dims& d, const float* q_mean, const f
 
 cudaError_t launch_route(const Dims& d, const float* q_mean, const float* k_mean,
                          int32_t* index, cudaStream_t st) {
+    // up to 64 regions, 32 channels per routing head, a few winners per row and enough (image, head) pairs for
+    // well over one 256-thread CTA per SM: one CTA per pair.  (Measured against the kernels below, route + pooling:
+    // 16.5 against 18.6 us at B = 64, 4 heads, k = 4; level at 512 pairs, k = 16; slower with 128 pairs, k = 1
+    // (18.6 against 17.5 us) and with 4 pairs (19.8 against 12.6 us), where one CTA's latency is all there is.)
+    if (d.R <= 64 && (d.heads_i == 1 ? d.C : d.d) == 32 && d.topk >= 2 && d.topk <= 8 &&
+        (long long)d.B * d.heads_i >= 256) {
+        cudaError_t e = launch_kernel(route_small_kernel, dim3(d.B * d.heads_i), dim3(ROUTE_S_THREADS), 0, st,
+                                      /*after_own_kernel=*/true, q_mean, k_mean, index, d);
+        count_launch();
+        return e;
+    }
     // many winners per row and enough (image, head) pairs to fill the GPU with 64-thread CTAs:
     // one thread per row
     if (d.topk > 8 && (long long)d.B * d.heads_i >= 256 && route_rows_smem(d) <= 100 * 1024) {

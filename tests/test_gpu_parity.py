@@ -124,6 +124,10 @@ def test_route_shared_and_odd_shapes(bra):
         # many winners per row and many (image, head) pairs: the thread-per-row routing kernel
         (BraConfig("k=12-many-pairs", 130, 8, 8, 64, 2, 4, 12, "bf16"), False),
         (BraConfig("k=9-shared-wide-rows", 256, 6, 6, 48, 3, 3, 9, "bf16"), True),
+        # a few winners per row, many pairs, 32 channels per routing head: one CTA per (image, head)
+        (BraConfig("cta-per-pair", 130, 14, 14, 64, 2, 7, 5, "bf16"), False),
+        (BraConfig("cta-per-pair-k=R", 160, 4, 6, 64, 2, 2, 4, "f32"), False),
+        (BraConfig("cta-per-pair-shared", 300, 6, 6, 32, 1, 3, 4, "f32"), True),
     ]
     for cfg, shared in cases:
         x = synthetic.make_inputs(cfg, seed=77)
@@ -156,6 +160,13 @@ def test_route_exact_ties_go_to_lower_region(bra):
     Q = torch.randn(256, 8, 8, 32, device="cuda")
     _, _, idx = bra.bra_route(p, Q, torch.ones_like(Q))
     assert (idx.cpu().numpy() == np.arange(10)).all()
+    # and through the kernel with one CTA per (image, head) (2 <= k <= 8, at least 256 pairs, 32 channels per head)
+    cfg = BraConfig("ties-cta-per-pair", 256, 8, 8, 32, 1, 4, 5, "f32")
+    p = problem_of(bra, cfg)
+    _, _, idx = bra.bra_route(p, Q, torch.ones_like(Q))
+    assert (idx.cpu().numpy() == np.arange(5)).all()
+    _, _, idx0 = bra.bra_route(p, torch.zeros_like(Q), torch.randn_like(Q))
+    assert (idx0.cpu().numpy() == np.arange(5)).all()
 
 
 # ------------------------------------------------------------------ attention
