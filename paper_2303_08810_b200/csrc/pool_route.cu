@@ -20,7 +20,6 @@ pool_kernel(const T* __restrict__ Q, const T* __restrict__ K,
             float* __restrict__ q_mean, float* __restrict__ k_mean, Dims dm) {
     constexpr int VEC = Vec<T>::n;
     extern __shared__ float part[];   // [ws][C]
-    pdl_launch_dependents();
     const int r = blockIdx.x, b = blockIdx.y;
     const int ry = r / dm.S, rx = r - ry * dm.S;
     const T* src = blockIdx.z == 0 ? Q : K;
@@ -56,6 +55,7 @@ pool_kernel(const T* __restrict__ Q, const T* __restrict__ K,
             *reinterpret_cast<float4*>(&part[it * VEC + i]) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
     }
     __syncthreads();
+    pdl_launch_dependents();          // this CTA's loads are done: the next kernel may be set up
     const float inv = 1.0f / (float)dm.n_r;
     for (int c = threadIdx.x; c < dm.C; c += blockDim.x) {
         float s = 0.f;
@@ -73,7 +73,6 @@ pool_split_kernel(const T* __restrict__ Q, const T* __restrict__ K,
                   float* __restrict__ q_mean, float* __restrict__ k_mean, Dims dm) {
     constexpr int VEC = Vec<T>::n;
     extern __shared__ float part[];   // [2][ws][C]
-    pdl_launch_dependents();
     const int r = blockIdx.x, b = blockIdx.y;
     const int ry = r / dm.S, rx = r - ry * dm.S;
     const T* src = blockIdx.z == 0 ? Q : K;
@@ -87,6 +86,7 @@ pool_split_kernel(const T* __restrict__ Q, const T* __restrict__ K,
     float v[4][VEC];
 #pragma unroll
     for (int u = 0; u < 4; ++u) load_row<VEC>(p + (size_t)u * row_elems, v[u]);
+    pdl_launch_dependents();          // this CTA's loads are out: the next kernel may be set up
     float acc[VEC];
 #pragma unroll
     for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
@@ -106,8 +106,73 @@ pool_split_kernel(const T* __restrict__ Q, const T* __restrict__ K,
     }
 }
 
+// Small square regions (1 x 1, 2 x 2 or 4 x 4 tokens): one CTA per (row of regions, tensor, image); thread = (region of
+// that row, 16-byte channel vector) sums all tokens of its region itself - column by column, the rows of a column
+// in order, the columns in order: the sums of pool_kernel, bit for bit - so nothing goes through shared memory
+// and a CTA moves a whole row of regions.  (One CTA per region is 6 272 CTAs of 64 threads and 2 KB each at the
+// stage-3 shape: the launch rate of CTAs, not HBM, sets its time.)
+template <typename T, int HS, int WS>
+__global__ void __launch_bounds__(512)
+pool_rows_kernel(const T* __restrict__ Q, const T* __restrict__ K,
+                 float* __restrict__ q_mean, float* __restrict__ k_mean, Dims dm) {
+    constexpr int VEC = Vec<T>::n;
+    const int ry = blockIdx.x, b = blockIdx.z;
+    const T* src = blockIdx.y == 0 ? Q : K;
+    float* dst = blockIdx.y == 0 ? q_mean : k_mean;
+    const int cvecs = dm.C / VEC;
+    const int rx = threadIdx.x / cvecs, cv = threadIdx.x - rx * cvecs;
+    if (rx >= dm.S) return;
+    const size_t row_elems = (size_t)dm.W * dm.C;
+    const T* p = src + ((size_t)b * dm.H + (size_t)ry * HS) * row_elems + (size_t)rx * dm.ws * dm.C + (size_t)cv * VEC;
+    // all HS x WS loads of the thread are issued before the first sum
+    float v[WS][HS][VEC];
+#pragma unroll
+    for (int x = 0; x < WS; ++x)
+#pragma unroll
+        for (int y = 0; y < HS; ++y) load_row<VEC>(p + (size_t)y * row_elems + (size_t)x * dm.C, v[x][y]);
+    // the next kernel may be set up from here on: this CTA's loads are out
+    pdl_launch_dependents();
+    float total[VEC];
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) total[i] = 0.f;
+#pragma unroll
+    for (int x = 0; x < WS; ++x) {
+        float col[VEC];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) col[i] = 0.f;
+#pragma unroll
+        for (int y = 0; y < HS; ++y)
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) col[i] += v[x][y][i];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) total[i] += col[i];
+    }
+    const float inv = 1.0f / (float)dm.n_r;
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) total[i] *= inv;
+    store_row<VEC>(dst + ((size_t)b * dm.R + (size_t)ry * dm.S + rx) * dm.C + (size_t)cv * VEC, total);
+}
+
+template <typename T>
+static cudaError_t launch_pool_rows(const Dims& d, const void* Q, const void* K, float* q_mean, float* k_mean,
+                                    cudaStream_t st) {
+    const int threads = (d.S * (d.C / Vec<T>::n) + 31) / 32 * 32;
+    const dim3 grid(d.S, 2, d.B);
+    const T* q = static_cast<const T*>(Q);
+    const T* k = static_cast<const T*>(K);
+    if (d.hs == 1) pool_rows_kernel<T, 1, 1><<<grid, threads, 0, st>>>(q, k, q_mean, k_mean, d);
+    else if (d.hs == 2) pool_rows_kernel<T, 2, 2><<<grid, threads, 0, st>>>(q, k, q_mean, k_mean, d);
+    else pool_rows_kernel<T, 4, 4><<<grid, threads, 0, st>>>(q, k, q_mean, k_mean, d);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_pool(const Dims& d, int dtype, const void* Q, const void* K,
                         float* q_mean, float* k_mean, cudaStream_t st) {
+    // small regions: a CTA per row of regions
+    if ((d.hs == 1 || d.hs == 2 || d.hs == 4) && d.ws == d.hs && d.S * (d.C / (dtype == BRA_BF16 ? 8 : 4)) <= 512 && d.B <= 65535)
+        return dtype == BRA_BF16 ? launch_pool_rows<__nv_bfloat16>(d, Q, K, q_mean, k_mean, st)
+                                 : launch_pool_rows<float>(d, Q, K, q_mean, k_mean, st);
     const int vec = dtype == BRA_BF16 ? 8 : 4;
     int items = d.ws * (d.C / vec);
     int threads = ((items < 256 ? items : 256) + 31) / 32 * 32;
@@ -162,7 +227,6 @@ __global__ void __launch_bounds__(256)
 route_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ index, Dims dm) {
     extern __shared__ float4 ks4[];             // [R][dc + 4] floats: rows 16-byte aligned, conflict-free;
     float* ks = reinterpret_cast<float*>(ks4);  // then this CTA's rows of Q^r, [8][dc]
-    pdl_launch_dependents();
     pdl_wait();                                  // the means come from the kernel before
     const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
     const int dc = dm.heads_i == 1 ? dm.C : dm.d;   // channels the affinity sums over (a multiple of 4)
@@ -183,6 +247,7 @@ route_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ ind
             *reinterpret_cast<float4*>(&qs[r * dc + 4 * c4]) = __ldcg(reinterpret_cast<const float4*>(qb + (size_t)r * dm.C) + c4);
     }
     __syncthreads();
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     for (int i = blockIdx.y * ROWS_PER_CTA + warp; i < dm.R && i < (int)(blockIdx.y + 1) * ROWS_PER_CTA; i += nwarps) {
         // lane l scores candidates l, l + 32, ...: channels in increasing order, one fp32 FMA each
@@ -291,7 +356,6 @@ __global__ void __launch_bounds__(ROUTE_S_THREADS)
 route_small_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ index, Dims dm) {
     __shared__ __align__(16) float ks[64 * ROUTE_S_LD];
     __shared__ uint32_t sc[64 * ROUTE_S_SC];
-    pdl_launch_dependents();
     pdl_wait();                                  // the means come from the kernel before
     const int tid = threadIdx.x;
     const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
@@ -310,6 +374,7 @@ route_small_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict
         for (int c4 = 0; c4 < 8; ++c4) qreg[c4] = __ldcg(qrow + c4);
     }
     __syncthreads();
+    pdl_launch_dependents();
     // ---- 2. scores of candidates q, q + 4, ..., two at a time ----
     for (int j0 = q; j0 < 64; j0 += 8) {
         const int j1 = j0 + 4;
@@ -383,7 +448,6 @@ __global__ void __launch_bounds__(ROUTE_T_ROWS)
 route_rows_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ index, Dims dm) {
     extern __shared__ float4 kt4[];             // [R][dc + 4] floats, then [R][64] score bits
     float* ks = reinterpret_cast<float*>(kt4);
-    pdl_launch_dependents();
     pdl_wait();                                  // the means come from the kernel before
     const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
     const int dc = dm.heads_i == 1 ? dm.C : dm.d;
@@ -398,6 +462,7 @@ route_rows_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict_
         *reinterpret_cast<float4*>(&ks[r * ld + 4 * c4]) = __ldcg(reinterpret_cast<const float4*>(kb + (size_t)r * dm.C) + c4);
     }
     __syncthreads();
+    pdl_launch_dependents();
     const int i = blockIdx.y * ROUTE_T_ROWS + threadIdx.x;
     if (i >= dm.R) return;
     const float4* qrow = reinterpret_cast<const float4*>(q_mean + ((size_t)b * dm.R + i) * dm.C + c0);
@@ -513,7 +578,6 @@ __global__ void __launch_bounds__(256)
 route_half_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict__ index, Dims dm) {
     extern __shared__ float4 kh4[];             // [R][dc + 4] floats, then this CTA's 16 rows of Q^r
     float* ks = reinterpret_cast<float*>(kh4);
-    pdl_launch_dependents();
     pdl_wait();                                  // the means come from the kernel before
     const int b = blockIdx.x / dm.heads_i, h = blockIdx.x % dm.heads_i;
     const int dc = dm.heads_i == 1 ? dm.C : dm.d;
@@ -535,6 +599,7 @@ route_half_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict_
             *reinterpret_cast<float4*>(&qs[r * dc + 4 * c4]) = __ldcg(reinterpret_cast<const float4*>(qb + (size_t)r * dm.C) + c4);
     }
     __syncthreads();
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31, l16 = lane & 15, half = lane >> 4;
     const int lrow = (threadIdx.x >> 5) * 2 + half;          // this half-warp's row of the CTA
     const int i = row0 + lrow;
