@@ -185,6 +185,7 @@ bwd_dq_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __r
     }
     cp_async_wait<0>();
     __syncthreads();
+    pdl_launch_dependents();          // this CTA's slices are resident: the dK/dV kernel may be set up beside it
 
     const int g = lane >> 2, tq = lane & 3;
     const float sl2 = dm.scale * 1.4426950408889634f;
@@ -298,15 +299,18 @@ bwd_dkv_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __
     img_load_slice(sbase + gm.off_b, reinterpret_cast<const uint8_t*>(dOg) + img_off, dm.N, tok_bytes, tid, nthreads);
     cp_async_commit();
     if (dm.lce) img_load_weights(smem + gm.off_w, lce_w + (size_t)h * 32 * 25, true, tid, nthreads);
+    // The copies above read inputs of the call and may run beside the dQ kernel (programmatic dependent launch);
+    // the inverse routing index and delta are that kernel's: read after the wait, with coherent loads.
+    pdl_wait();
     // inverse routing index of this (image, head): offsets, then the query regions as token ids
     int32_t* s_off = reinterpret_cast<int32_t*>(smem + gm.off_idx);
     int32_t* s_list = s_off + dm.R + 1;
     {
         const int hi = dm.heads_i == 1 ? 0 : h;
         const size_t bh = (size_t)b * dm.heads_i + hi;
-        for (int e = tid; e <= dm.R; e += nthreads) s_off[e] = __ldg(inv_off + bh * (dm.R + 1) + e);
+        for (int e = tid; e <= dm.R; e += nthreads) s_off[e] = __ldcg(inv_off + bh * (dm.R + 1) + e);
         for (int e = tid; e < dm.R * dm.topk; e += nthreads) {
-            int r = __ldg(inv_list + bh * dm.R * dm.topk + e);
+            int r = __ldcg(inv_list + bh * dm.R * dm.topk + e);
             r = min(max(r, 0), dm.R - 1);              // entries past the last list are never read
             const int qy = fdiv(r, dm.S, gm.mul_s), qx = r - qy * dm.S;
             s_list[e] = qy * dm.hs * dm.W + qx * dm.ws;
@@ -353,7 +357,7 @@ bwd_dkv_img_kernel(const __nv_bfloat16* __restrict__ Qg, const __nv_bfloat16* __
             for (int e = 0; e < 2; ++e) {
                 const bool valid = (vm[e] >> lane) & 1u;
                 cl[e] = valid ? __ldg(lse + stat0 + (trow[e] >> 6)) * 1.4426950408889634f : 0.f;   // >> 6: the token
-                cd[e] = valid ? __ldg(delta + stat0 + (trow[e] >> 6)) : 0.f;
+                cd[e] = valid ? __ldcg(delta + stat0 + (trow[e] >> 6)) : 0.f;
             }
             float c[8][4], dp[8][4];
             img_rows_x_gather_t2(c, ka, qbase, dp, va, gbase, trow, lane);   // S^T = K Q^T, dP^T = V dO^T
@@ -493,11 +497,11 @@ cudaError_t launch_backward_img(const Dims& d, const void* Q, const void* K, con
                                                                     const_cast<int32_t*>(inv_list), status, d, a);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    dkv_kernel<<<(unsigned)grid, b.nw * 32, b.smem_bytes, st>>>(q, k, v, inv_off, inv_list, lse, delta, go, lce_w,
-                                                                     static_cast<__nv_bfloat16*>(dK),
-                                                                     static_cast<__nv_bfloat16*>(dV), d, b);
+    e = launch_kernel(dkv_kernel, dim3((unsigned)grid), dim3(b.nw * 32), (size_t)b.smem_bytes, st, /*after_own_kernel=*/true,
+                      q, k, v, inv_off, inv_list, lse, static_cast<const float*>(delta), go, lce_w,
+                      static_cast<__nv_bfloat16*>(dK), static_cast<__nv_bfloat16*>(dV), d, b);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace bra
