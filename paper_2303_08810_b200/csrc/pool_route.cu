@@ -373,10 +373,11 @@ route_small_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict
 #pragma unroll
         for (int c4 = 0; c4 < 8; ++c4) qreg[c4] = __ldcg(qrow + c4);
     }
+    for (int e = tid; e < 64 * ROUTE_S_SC; e += ROUTE_S_THREADS) sc[e] = 0u;     // 0: no candidate
     __syncthreads();
     pdl_launch_dependents();
     // ---- 2. scores of candidates q, q + 4, ..., two at a time ----
-    for (int j0 = q; j0 < 64; j0 += 8) {
+    for (int j0 = q; j0 < dm.R; j0 += 8) {
         const int j1 = j0 + 4;
         const float4* ka = reinterpret_cast<const float4*>(&ks[(j0 < dm.R ? j0 : 0) * ROUTE_S_LD]);
         const float4* kb4 = reinterpret_cast<const float4*>(&ks[(j1 < dm.R ? j1 : 0) * ROUTE_S_LD]);
@@ -390,8 +391,8 @@ route_small_kernel(const float* q_mean, const float* k_mean, int32_t* __restrict
             a0 = fmaf(qreg[c4].w, x.w, a0); a1 = fmaf(qreg[c4].w, y.w, a1);
         }
         // 0 marks "no candidate": real score bits are never 0
-        sc[i * ROUTE_S_SC + j0] = j0 < dm.R ? ordered_bits(a0) : 0u;
-        sc[i * ROUTE_S_SC + j1] = j1 < dm.R ? ordered_bits(a1) : 0u;
+        sc[i * ROUTE_S_SC + j0] = ordered_bits(a0);
+        if (j1 < dm.R) sc[i * ROUTE_S_SC + j1] = ordered_bits(a1);
     }
     __syncthreads();
     // ---- 3. selection, one thread per row (the other warps are done) ----
@@ -686,11 +687,12 @@ static cudaError_t launch_route_rows(const Dims& d, const float* q_mean, const f
 
 cudaError_t launch_route(const Dims& d, const float* q_mean, const float* k_mean,
                          int32_t* index, cudaStream_t st) {
-    // up to 64 regions, 32 channels per routing head, a few winners per row and enough (image, head) pairs for
-    // well over one 256-thread CTA per SM: one CTA per pair.  (Measured against the kernels below, route + pooling:
-    // 16.5 against 18.6 us at B = 64, 4 heads, k = 4; level at 512 pairs, k = 16; slower with 128 pairs, k = 1
-    // (18.6 against 17.5 us) and with 4 pairs (19.8 against 12.6 us), where one CTA's latency is all there is.)
-    if (d.R <= 64 && (d.heads_i == 1 ? d.C : d.d) == 32 && d.topk >= 2 && d.topk <= 8 &&
+    // up to 64 regions, 32 channels per routing head, more than one winner per row and enough (image, head)
+    // pairs for well over one 256-thread CTA per SM: one CTA per pair.  (Measured against the kernels below,
+    // pooling + routing: 14.5 against 15.8 us at B = 64, 4 heads, k = 4; 18.6 against 20.6 us at 512 pairs,
+    // k = 16; slower with 128 pairs, k = 1 (18.6 against 17.5 us) and with 4 pairs (19.8 against 12.6 us),
+    // where one CTA's latency is all there is.)
+    if (d.R <= 64 && (d.heads_i == 1 ? d.C : d.d) == 32 && d.topk >= 2 &&
         (long long)d.B * d.heads_i >= 256) {
         cudaError_t e = launch_kernel(route_small_kernel, dim3(d.B * d.heads_i), dim3(ROUTE_S_THREADS), 0, st,
                                       /*after_own_kernel=*/true, q_mean, k_mean, index, d);
