@@ -124,6 +124,10 @@ def test_route_shared_and_odd_shapes(bra):
         # many winners per row and many (image, head) pairs: the thread-per-row routing kernel
         (BraConfig("k=12-many-pairs", 130, 8, 8, 64, 2, 4, 12, "bf16"), False),
         (BraConfig("k=9-shared-wide-rows", 256, 6, 6, 48, 3, 3, 9, "bf16"), True),
+        # small square regions: pooled by one CTA per row of regions
+        (BraConfig("1x1-regions", 3, 5, 5, 64, 2, 5, 7, "bf16"), False),
+        (BraConfig("2x2-regions-f32", 2, 8, 8, 32, 1, 4, 3, "f32"), False),
+        (BraConfig("4x4-regions-wide-rows", 2, 12, 12, 512, 16, 3, 2, "bf16"), True),
         # a few winners per row, many pairs, 32 channels per routing head: one CTA per (image, head)
         (BraConfig("cta-per-pair", 130, 14, 14, 64, 2, 7, 5, "bf16"), False),
         (BraConfig("cta-per-pair-k=R", 160, 4, 6, 64, 2, 2, 4, "f32"), False),
