@@ -86,7 +86,6 @@ pool_split_kernel(const T* __restrict__ Q, const T* __restrict__ K,
     float v[4][VEC];
 #pragma unroll
     for (int u = 0; u < 4; ++u) load_row<VEC>(p + (size_t)u * row_elems, v[u]);
-    pdl_launch_dependents();          // this CTA's loads are out: the next kernel may be set up
     float acc[VEC];
 #pragma unroll
     for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
@@ -98,6 +97,7 @@ pool_split_kernel(const T* __restrict__ Q, const T* __restrict__ K,
     for (int i = 0; i < VEC; i += 4)
         *reinterpret_cast<float4*>(&part[yh * wsC + it * VEC + i]) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
     __syncthreads();
+    pdl_launch_dependents();          // this CTA's loads are done: the next kernel may be set up
     const float inv = 1.0f / (float)dm.n_r;
     for (int c = threadIdx.x; c < dm.C; c += blockDim.x) {
         float s = 0.f;
